@@ -1,0 +1,165 @@
+"""fp64 CPU oracle for low-rank pre-factorized layers -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package.  It shares no code with the CUDA library and never imports it.  The arithmetic
+lives in ``pf_oracle.c`` (plain loops in double precision, one per definition); this file
+only widens stored inputs to fp64 exactly, marshals numpy arrays and defines the
+comparison metric.
+
+Functions (paper passages they follow are cited in ``pf_oracle.c``):
+
+    linear_fwd(x, U, V)              -> y, T            y = (x U) V^T
+    linear_bwd(x, U, V, dY)          -> dX, dU, dV      chain rule on the above
+    conv_fwd(x, U, V, stride, pad)   -> y, T            k x k conv to r channels, then 1 x 1
+    conv_bwd(x, U, V, dY, stride, pad) -> dX, dU, dV
+    pack(list_of_arrays)             -> flat, offsets   flat gradient buffer
+
+Parity pins (tests/test_oracle_*.py): hand-computed tiny cases, the dense identity
+(xU)V^T = x(UV^T), special cases that reduce to a textbook matrix product or a library
+correlation, the dense chain rule, central finite differences, an independent
+im2col route for the convolution, Table 1 parameter counts and pure-Python brute force.
+The paper prints no numeric layer output, so no output value is pinned by its text.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libpf_oracle.so")
+_SRC = os.path.join(_HERE, "pf_oracle.c")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile pf_oracle.c with gcc (OpenMP) into libpf_oracle.so next to it."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+                               "-o", tmp, _SRC])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_SO)
+        L, D, I = ctypes.c_long, ctypes.c_void_p, ctypes.c_int
+        lib.pf_oracle_threads.restype = I
+        lib.pf_oracle_linear_fwd.argtypes = [D, D, D, L, L, L, L, D, D]
+        lib.pf_oracle_linear_bwd.argtypes = [D, D, D, D, D, L, L, L, L, D, D, D, D]
+        lib.pf_oracle_conv_fwd.argtypes = [D, D, D] + [L] * 10 + [D, D]
+        lib.pf_oracle_conv_bwd.argtypes = [D, D, D, D, D] + [L] * 10 + [D, D, D, D]
+        lib.pf_oracle_pack.argtypes = [D, D, I, I, D, D]
+        for f in ("linear_fwd", "linear_bwd", "conv_fwd", "conv_bwd", "pack"):
+            getattr(lib, "pf_oracle_" + f).restype = None
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    return int(_load().pf_oracle_threads())
+
+
+def widen(a) -> np.ndarray:
+    """Stored values -> float64, exactly.  uint16 arrays are bf16 bit patterns."""
+    a = np.asarray(a)
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def linear_fwd(x, U, V):
+    x, U, V = widen(x), widen(U), widen(V)
+    m, k = x.shape
+    k2, r = U.shape
+    n, r2 = V.shape
+    assert k == k2 and r == r2
+    T = np.empty((m, r))
+    y = np.empty((m, n))
+    _load().pf_oracle_linear_fwd(_p(x), _p(U), _p(V), m, k, n, r, _p(T), _p(y))
+    return y, T
+
+
+def linear_bwd(x, U, V, dY):
+    x, U, V, dY = widen(x), widen(U), widen(V), widen(dY)
+    m, k = x.shape
+    n, r = V.shape
+    assert U.shape == (k, r) and dY.shape == (m, n)
+    _, T = linear_fwd(x, U, V)
+    G = np.empty((m, r))
+    dX = np.empty((m, k))
+    dU = np.empty((k, r))
+    dV = np.empty((n, r))
+    _load().pf_oracle_linear_bwd(_p(x), _p(U), _p(V), _p(dY), _p(T), m, k, n, r,
+                                 _p(G), _p(dX), _p(dU), _p(dV))
+    return dX, dU, dV
+
+
+def conv_out_hw(H, W, kh, kw, stride, pad):
+    return (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
+
+
+def conv_fwd(x, U, V, stride=1, pad=1):
+    x, U, V = widen(x), widen(U), widen(V)
+    N, H, W, C = x.shape
+    kh, kw, C2, R = U.shape
+    O, R2 = V.shape
+    assert C == C2 and R == R2
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad)
+    T = np.empty((N, Ho, Wo, R))
+    y = np.empty((N, Ho, Wo, O))
+    _load().pf_oracle_conv_fwd(_p(x), _p(U), _p(V), N, H, W, C, R, O, kh, kw, stride, pad,
+                               _p(T), _p(y))
+    return y, T
+
+
+def conv_bwd(x, U, V, dY, stride=1, pad=1):
+    x, U, V, dY = widen(x), widen(U), widen(V), widen(dY)
+    N, H, W, C = x.shape
+    kh, kw, _, R = U.shape
+    O = V.shape[0]
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad)
+    assert dY.shape == (N, Ho, Wo, O)
+    _, T = conv_fwd(x, U, V, stride, pad)
+    dT = np.empty((N, Ho, Wo, R))
+    dX = np.empty((N, H, W, C))
+    dU = np.empty((kh, kw, C, R))
+    dV = np.empty((O, R))
+    _load().pf_oracle_conv_bwd(_p(x), _p(U), _p(V), _p(dY), _p(T), N, H, W, C, R, O,
+                               kh, kw, stride, pad, _p(dT), _p(dX), _p(dU), _p(dV))
+    return dX, dU, dV
+
+
+def pack(grads):
+    """Flat gradient buffer: values copied bit for bit, in list order, tightly."""
+    grads = [np.ascontiguousarray(g).reshape(-1) for g in grads]
+    count = len(grads)
+    dt = grads[0].dtype if count else np.dtype(np.uint16)
+    assert all(g.dtype == dt for g in grads)
+    numels = np.array([g.size for g in grads], dtype=np.int64)
+    total = int(numels.sum())
+    flat = np.empty(total, dtype=dt)
+    offsets = np.zeros(count + 1, dtype=np.int64)
+    ptrs = (ctypes.c_void_p * max(count, 1))(*[g.ctypes.data for g in grads])
+    _load().pf_oracle_pack(ctypes.cast(ptrs, ctypes.c_void_p), _p(numels), count,
+                           dt.itemsize, _p(flat), _p(offsets))
+    return flat, offsets
+
+
+def rel_err(z, z_ref) -> float:
+    """Frobenius-norm-relative error  ||z - z_ref||_F / max(||z_ref||_F, tiny)  in fp64."""
+    z = widen(z).reshape(-1)
+    z_ref = np.asarray(z_ref, dtype=np.float64).reshape(-1)
+    assert z.shape == z_ref.shape, (z.shape, z_ref.shape)
+    den = max(float(np.linalg.norm(z_ref)), 1e-300)
+    return float(np.linalg.norm(z - z_ref)) / den

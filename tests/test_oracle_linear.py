@@ -1,0 +1,126 @@
+"""Pins for the fp64 oracle of the factorized FC layer (Section 2.1, Appendix B "FC layer").
+
+None of these re-type the oracle's own loops: they check it against a hand-computed
+example, the dense identity, textbook special cases, the dense chain rule, finite
+differences and pure-Python brute force of the index definition.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from _util import read_golden, rng_int
+
+
+def test_hand_case(golden_dir):
+    g = read_golden(os.path.join(golden_dir, "linear_hand_case.txt"))
+    y, T = oracle.linear_fwd(g["x"], g["U"], g["V"])
+    dX, dU, dV = oracle.linear_bwd(g["x"], g["U"], g["V"], g["dY"])
+    for got, want in ((y, "y"), (T, "T"), (dX, "dX"), (dU, "dU"), (dV, "dV")):
+        np.testing.assert_array_equal(got, g[want])
+
+
+@pytest.mark.parametrize("m,k,n,r", [(1, 1, 1, 1), (5, 7, 3, 2), (4, 3, 9, 5), (13, 6, 2, 11)])
+def test_fwd_dense_identity(m, k, n, r):
+    """(xU)V^T = x(UV^T): W ~ U V^T is the whole point of Section 2.1."""
+    x, U, V = rng_int(1, (m, k)), rng_int(2, (k, r)), rng_int(3, (n, r))
+    y, T = oracle.linear_fwd(x, U, V)
+    np.testing.assert_array_equal(y, x @ (U @ V.T))
+    np.testing.assert_array_equal(T, x @ U)
+
+
+def test_fwd_dense_identity_real_values():
+    rng = np.random.default_rng(0)
+    x, U, V = rng.normal(size=(17, 23)), rng.normal(size=(23, 5)), rng.normal(size=(11, 5))
+    y, _ = oracle.linear_fwd(x, U, V)
+    assert oracle.rel_err(y, x @ (U @ V.T)) < 1e-13
+
+
+def test_fwd_identity_factor_is_plain_matmul():
+    """r = k and U = I reduces the layer to the textbook product x V^T."""
+    x, V = rng_int(4, (6, 5)), rng_int(5, (8, 5))
+    y, T = oracle.linear_fwd(x, np.eye(5), V)
+    np.testing.assert_array_equal(y, x @ V.T)
+    np.testing.assert_array_equal(T, x)
+
+
+def test_fwd_brute_force_python_loops():
+    m, k, n, r = 3, 4, 5, 2
+    x, U, V = rng_int(6, (m, k)), rng_int(7, (k, r)), rng_int(8, (n, r))
+    want = np.zeros((m, n))
+    for i in range(m):
+        for o in range(n):
+            for j in range(r):
+                for c in range(k):
+                    want[i, o] += x[i, c] * U[c, j] * V[o, j]
+    y, _ = oracle.linear_fwd(x, U, V)
+    np.testing.assert_array_equal(y, want)
+
+
+@pytest.mark.parametrize("m,k,n,r", [(5, 7, 3, 2), (4, 3, 9, 5), (2, 6, 6, 8)])
+def test_bwd_dense_chain_rule(m, k, n, r):
+    """Dense layer y = xW, W = UV^T: dW = x^T dY, dX = dY W^T, then dU = dW V, dV = dW^T U."""
+    x, U, V, dY = (rng_int(10, (m, k)), rng_int(11, (k, r)), rng_int(12, (n, r)),
+                   rng_int(13, (m, n)))
+    dX, dU, dV = oracle.linear_bwd(x, U, V, dY)
+    W = U @ V.T
+    dW = x.T @ dY
+    np.testing.assert_array_equal(dX, dY @ W.T)
+    np.testing.assert_array_equal(dU, dW @ V)
+    np.testing.assert_array_equal(dV, dW.T @ U)
+
+
+def test_bwd_finite_differences():
+    """L = sum(dY * y); central differences in every entry of x, U, V."""
+    rng = np.random.default_rng(3)
+    m, k, n, r = 4, 5, 6, 3
+    x, U, V, dY = (rng.normal(size=(m, k)), rng.normal(size=(k, r)), rng.normal(size=(n, r)),
+                   rng.normal(size=(m, n)))
+    dX, dU, dV = oracle.linear_bwd(x, U, V, dY)
+
+    def loss(x_, U_, V_):
+        return float(np.sum(dY * oracle.linear_fwd(x_, U_, V_)[0]))
+
+    h = 1e-6
+    for arr, grad, idx in ((x, dX, 0), (U, dU, 1), (V, dV, 2)):
+        fd = np.zeros_like(arr)
+        for pos in np.ndindex(arr.shape):
+            args = [x.copy(), U.copy(), V.copy()]
+            args[idx][pos] += h
+            up = loss(*args)
+            args[idx][pos] -= 2 * h
+            dn = loss(*args)
+            fd[pos] = (up - dn) / (2 * h)
+        assert oracle.rel_err(grad, fd) < 1e-7
+
+
+def test_bwd_is_plain_sum_over_rows_no_mean():
+    """Stacking the same batch twice doubles dU and dV (no 1/m anywhere)."""
+    x, U, V, dY = rng_int(20, (3, 4)), rng_int(21, (4, 2)), rng_int(22, (5, 2)), rng_int(23, (3, 5))
+    _, dU1, dV1 = oracle.linear_bwd(x, U, V, dY)
+    _, dU2, dV2 = oracle.linear_bwd(np.vstack([x, x]), U, V, np.vstack([dY, dY]))
+    np.testing.assert_array_equal(dU2, 2 * dU1)
+    np.testing.assert_array_equal(dV2, 2 * dV1)
+
+
+def test_rank_column_slicing_gives_matching_gradient_columns():
+    """dU[:, J] and dV[:, J] only depend on columns J of U and V: this is what lets
+    full-size parity checks sample the factor gradients."""
+    x, U, V, dY = rng_int(30, (6, 5)), rng_int(31, (5, 4)), rng_int(32, (7, 4)), rng_int(33, (6, 7))
+    _, dU, dV = oracle.linear_bwd(x, U, V, dY)
+    J = [1, 3]
+    _, dUj, dVj = oracle.linear_bwd(x, U[:, J], V[:, J], dY)
+    np.testing.assert_array_equal(dUj, dU[:, J])
+    np.testing.assert_array_equal(dVj, dV[:, J])
+
+
+def test_widen_bf16_bits_exact():
+    bits = np.array([0x3F80, 0xBF80, 0x4000, 0x3F00, 0x0000, 0x3FC0], dtype=np.uint16)
+    np.testing.assert_array_equal(oracle.widen(bits), [1.0, -1.0, 2.0, 0.5, 0.0, 1.5])
+
+
+def test_rel_err_metric():
+    a = np.array([3.0, 4.0])
+    assert oracle.rel_err(a, a) == 0.0
+    assert abs(oracle.rel_err(a + np.array([0.3, 0.4]), a) - 0.1) < 1e-15
