@@ -1,0 +1,156 @@
+/*
+ * pf.h -- C ABI of the low-rank pre-factorized layer library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the forward and backward passes of layers whose dense weight
+ * W (k x n) has been replaced by two factors U (k x r) and V (n x r), W ~ U V^T
+ * (Pufferfish, Section 2), plus the flat gradient buffer that is communicated once per
+ * iteration (Section 4.1).
+ *
+ * Conventions common to every entry point
+ *   - All tensor pointers are DEVICE pointers unless a parameter says "host".
+ *   - The caller owns every buffer.  The library never allocates, frees or
+ *     synchronises; all work is enqueued on `cuda_stream` (a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream) and returns immediately.
+ *   - Inputs are never modified.  Outputs are overwritten (never accumulated into).
+ *     No output may alias an input or another output.
+ *   - All tensors of one call share `dtype`; products are accumulated in fp32 and
+ *     rounded once (round-to-nearest-even) to `dtype` at the final store.  With
+ *     PF_BF16 the on-chip intermediate x U (and dY V) is rounded to bf16 before the
+ *     second product.
+ *   - Matrices are row-major.  A leading dimension `ld*` is the distance in ELEMENTS
+ *     between consecutive rows and must be >= the row length.
+ *   - `workspace` is caller-provided scratch of at least the matching
+ *     pf_*_workspace() query, 256-byte aligned; its contents are undefined afterwards.
+ *     Two calls that may overlap on the GPU must not share a workspace.
+ *   - Every entry returns a pf_status.  Errors detected on the host (bad pointer,
+ *     bad dimension, workspace too small, ...) are returned BEFORE anything is
+ *     launched.  Nothing is printed, nothing aborts.
+ *   - Problems with no rows / no tensors (m = 0, N = 0, count = 0) are PF_OK no-ops.
+ */
+#ifndef PF_H_
+#define PF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PF_OK = 0,
+    PF_ERR_INVALID_ARG = 1, /* null required pointer, dimension < 1, ld too small, bad dtype,
+                               misaligned pointer, negative count */
+    PF_ERR_UNSUPPORTED = 2, /* valid mathematics outside the implemented envelope */
+    PF_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small; pack capacity too small */
+    PF_ERR_CUDA = 4,        /* a CUDA runtime / driver call or a launch failed */
+    PF_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (see pf_last_device_status) */
+} pf_status;
+
+typedef enum {
+    PF_F32 = 0, /* fp32 storage, fp32 FMA arithmetic */
+    PF_BF16 = 1 /* bf16 storage, tensor-core products with fp32 accumulation */
+} pf_dtype;
+
+/* Static, human-readable name of a status code. */
+const char* pf_status_string(int status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int pf_version(void);
+
+/* Number of kernels this library has launched in this process so far (monotonic, all
+ * devices and streams).  Lets a caller verify that work ran in this library's kernels. */
+long long pf_launch_count(void);
+
+/* Device-side status of the current device: PF_OK, or PF_ERR_TIMEOUT if a kernel of
+ * this library gave up on a bounded wait since the last query.  Synchronises the
+ * device (blocking) and clears the flag.  Never needed on the normal path. */
+int pf_last_device_status(void);
+
+/* ---------------------------------------------------------------------------------
+ * Factorized fully-connected layer   y = (x U) V^T
+ * (Section 2.1 "Low-rank factorization for FC layers"; Appendix B "FC layer", whose
+ *  row convention (xU)V^T is used: U is the input-side factor, V the output-side one.)
+ *
+ *   x [m, k] (ldx)   U [k, r] (ldu)   V [n, r] (ldv)   y [m, n] (ldy)
+ *   T_stash [m, r] (ldt): optional output, the intermediate T = x U rounded to `dtype`,
+ *                         for reuse by the backward pass; NULL = not written.
+ * m >= 0; k, n, r >= 1 (r need not divide anything; r > min(k, n) is legal).
+ * ------------------------------------------------------------------------------- */
+size_t pf_lowrank_linear_workspace(int64_t m, int64_t k, int64_t n, int64_t r,
+                                   int dtype, int is_bwd);
+
+int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu,
+                          const void* V, int64_t ldv, void* y, int64_t ldy,
+                          void* T_stash, int64_t ldt,
+                          int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Gradients of the layer above for an upstream gradient dY [m, n] (chain rule on
+ * y = (xU)V^T; plain sums over the m rows, no averaging):
+ *   G  = dY V           [m, r]  (kept on chip / in workspace)
+ *   dX = G U^T          [m, k]  (lddx)   NULL = not wanted (first layer)
+ *   dU = x^T G          [k, r]  (lddu)
+ *   dV = dY^T (x U)     [n, r]  (lddv)
+ * T_stash [m, r] (ldt): the forward's stashed x U, or NULL to have it recomputed. */
+int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu,
+                          const void* V, int64_t ldv, const void* dY, int64_t lddy,
+                          const void* T_stash, int64_t ldt,
+                          void* dX, int64_t lddx, void* dU, int64_t lddu, void* dV, int64_t lddv,
+                          int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------
+ * Factorized convolution: a kh x kw convolution into R channels (factor U) followed by a
+ * 1 x 1 convolution to O channels (factor V), nothing in between
+ * (Section 2.2 "Factorizing a convolution layer"; Appendix B "Convolution layer").
+ * Cross-correlation (no kernel flip), zero padding `pad`, stride `stride` on the
+ * kh x kw convolution only; no dilation, no groups.
+ *
+ *   x [N, H, W, C] NHWC, contiguous
+ *   U [kh, kw, C, R]  = the unrolled (kh*kw*C) x R matrix of Section 2.2, rows tap-major
+ *   V [O, R]
+ *   y [N, Ho, Wo, O] NHWC,  Ho = (H + 2 pad - kh) / stride + 1 (floor), Wo likewise
+ *   T_stash [N, Ho, Wo, R]: optional output of the thin convolution; NULL = not written.
+ * Returns PF_ERR_UNSUPPORTED for kh != kw or stride < 1.
+ * ------------------------------------------------------------------------------- */
+size_t pf_lowrank_conv_workspace(int N, int H, int W, int C, int R, int O,
+                                 int kh, int kw, int stride, int pad, int dtype, int is_bwd);
+
+int pf_lowrank_conv_fwd(const void* x, const void* U, const void* V, void* y, void* T_stash,
+                        int N, int H, int W, int C, int R, int O,
+                        int kh, int kw, int stride, int pad, int dtype,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Gradients of the factorized convolution for dY [N, Ho, Wo, O]:
+ *   dT = dY V (per pixel), dV [O, R] = dY^T T, dU [kh, kw, C, R] = im2col(x)^T dT,
+ *   dX [N, H, W, C] = transposed convolution of dT with U (NULL = not wanted).
+ * T_stash: the forward's stash or NULL to recompute. */
+int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void* dY,
+                        const void* T_stash, void* dX, void* dU, void* dV,
+                        int N, int H, int W, int C, int R, int O,
+                        int kh, int kw, int stride, int pad, int dtype,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------
+ * Flat gradient buffer (Section 4.1 "Implementation details and optimizations": all
+ * gradient tensors are packed into one flat buffer so that one all-reduce per iteration
+ * suffices).  Copies tensor i (numels[i] elements of `dtype`) bit for bit to
+ * flat[offsets_out[i] ...], in list order, tightly (no padding, no conversion, no scaling):
+ *   offsets_out[0] = 0, offsets_out[i+1] = offsets_out[i] + numels[i].
+ *
+ *   grads        host array of `count` device pointers (element-aligned)
+ *   numels       host array of `count` element counts (>= 0)
+ *   flat         device buffer of `flat_capacity_elems` elements
+ *   offsets_out  host array of count+1 entries, written before return (element units)
+ * No workspace is needed (workspace arguments are accepted and ignored).
+ * PF_ERR_WORKSPACE if the tensors do not fit in flat_capacity_elems.
+ * ------------------------------------------------------------------------------- */
+int pf_pack_factor_grads(const void* const* grads, const int64_t* numels, int count, int dtype,
+                         void* flat, int64_t flat_capacity_elems, int64_t* offsets_out,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PF_H_ */

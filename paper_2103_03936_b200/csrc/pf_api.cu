@@ -1,0 +1,425 @@
+// C-ABI entry points of libpf: argument validation, workspace layout, path selection
+// (tensor-core kernels for bf16 inside their envelope, FMA kernels otherwise) and launches.
+// Nothing here allocates or synchronises; see include/pf.h for the contract.
+#include <atomic>
+#include <cstring>
+
+#include "pf_internal.h"
+#include "pf_tc.h"
+
+namespace pf {
+namespace {
+
+__device__ unsigned int g_device_status;  // 0 = fine; kernels store a PF_ERR_* code here
+
+struct PerDevice {
+    unsigned int* status_ptr;
+    bool ready;
+};
+PerDevice g_dev[64];
+
+bool elem_aligned(const void* p, int dtype) {
+    return (reinterpret_cast<uintptr_t>(p) % dtype_size(dtype)) == 0;
+}
+bool valid_dtype(int dtype) { return dtype == PF_F32 || dtype == PF_BF16; }
+
+int check_ws(const void* ws, size_t have, size_t need) {
+    if (need == 0) return PF_OK;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || have < need)
+        return PF_ERR_WORKSPACE;
+    return PF_OK;
+}
+
+#define PF_CUDA(expr)                                   \
+    do {                                                \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) return PF_ERR_CUDA;     \
+    } while (0)
+
+MatA plainA(const void* p, int64_t s_row, int64_t s_col) {
+    MatA a;
+    std::memset(&a, 0, sizeof(a));
+    a.p = p; a.s_row = s_row; a.s_col = s_col; a.kind = A_PLAIN; a.l_fast = (s_col == 1);
+    return a;
+}
+MatB plainB(const void* p, int64_t s_row, int64_t s_col) {
+    MatB b;
+    std::memset(&b, 0, sizeof(b));
+    b.p = p; b.s_row = s_row; b.s_col = s_col; b.kind = B_PLAIN; b.l_fast = (s_col != 1);
+    return b;
+}
+SimtGemm mk(const MatA& A, const MatB& B, void* C, int64_t ldc, int64_t M, int64_t N, int64_t K,
+            int dtype, int splits = 1, float* partial = nullptr) {
+    SimtGemm g;
+    g.A = A; g.B = B; g.C = C; g.ldc = ldc; g.M = M; g.N = N; g.K = K;
+    g.splits = splits; g.partial = partial; g.dtype = dtype;
+    return g;
+}
+
+// ------------------------------------------------------------------------------ linear
+struct LinearWs {
+    size_t off_T, off_G, off_partial, off_tc, total;
+    int splits_dU, splits_dV;
+};
+
+LinearWs linear_ws(int64_t m, int64_t k, int64_t n, int64_t r, int dtype, bool bwd) {
+    LinearWs w;
+    std::memset(&w, 0, sizeof(w));
+    const size_t s = dtype_size(dtype);
+    size_t off = 0;
+    w.off_T = off; off += align_up(static_cast<size_t>(m) * r * s, 256);
+    if (bwd) {
+        w.off_G = off; off += align_up(static_cast<size_t>(m) * r * s, 256);
+        w.splits_dU = simt_pick_splits(k, r, m);
+        w.splits_dV = simt_pick_splits(n, r, m);
+        size_t pu = w.splits_dU > 1 ? static_cast<size_t>(w.splits_dU) * k * r * 4 : 0;
+        size_t pv = w.splits_dV > 1 ? static_cast<size_t>(w.splits_dV) * n * r * 4 : 0;
+        w.off_partial = off; off += align_up(pu > pv ? pu : pv, 256);
+    }
+    w.off_tc = off;
+    if (dtype == PF_BF16) off += align_up(tc::linear_extra_workspace(m, k, n, r, bwd), 256);
+    w.total = off;
+    return w;
+}
+
+int validate_linear_common(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
+                           int64_t ldv, int64_t m, int64_t k, int64_t n, int64_t r, int dtype) {
+    if (!valid_dtype(dtype)) return PF_ERR_INVALID_ARG;
+    if (m < 0 || k < 1 || n < 1 || r < 1) return PF_ERR_INVALID_ARG;
+    if (!x || !U || !V) return PF_ERR_INVALID_ARG;
+    if (ldx < k || ldu < r || ldv < r) return PF_ERR_INVALID_ARG;
+    if (!elem_aligned(x, dtype) || !elem_aligned(U, dtype) || !elem_aligned(V, dtype))
+        return PF_ERR_INVALID_ARG;
+    if (m > (1LL << 40) || k > (1LL << 31) || n > (1LL << 31) || r > (1LL << 20)) return PF_ERR_UNSUPPORTED;
+    return PF_OK;
+}
+
+}  // namespace
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
+
+unsigned int* device_status_ptr() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!g_dev[dev].ready) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        g_dev[dev].status_ptr = static_cast<unsigned int*>(p);
+        g_dev[dev].ready = true;
+    }
+    return g_dev[dev].status_ptr;
+}
+
+}  // namespace pf
+
+using namespace pf;
+
+extern "C" {
+
+const char* pf_status_string(int status) {
+    switch (status) {
+        case PF_OK: return "PF_OK";
+        case PF_ERR_INVALID_ARG: return "PF_ERR_INVALID_ARG";
+        case PF_ERR_UNSUPPORTED: return "PF_ERR_UNSUPPORTED";
+        case PF_ERR_WORKSPACE: return "PF_ERR_WORKSPACE";
+        case PF_ERR_CUDA: return "PF_ERR_CUDA";
+        case PF_ERR_TIMEOUT: return "PF_ERR_TIMEOUT";
+        default: return "PF_ERR_UNKNOWN";
+    }
+}
+
+int pf_version(void) { return 100; }
+
+long long pf_launch_count(void) { return launches_so_far(); }
+
+int pf_last_device_status(void) {
+    unsigned int* p = device_status_ptr();
+    if (!p) return PF_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PF_ERR_CUDA;
+    unsigned int v = 0;
+    if (cudaMemcpy(&v, p, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return PF_ERR_CUDA;
+    if (v != 0) {
+        const unsigned int zero = 0;
+        if (cudaMemcpy(p, &zero, sizeof(zero), cudaMemcpyHostToDevice) != cudaSuccess) return PF_ERR_CUDA;
+    }
+    return v == 0 ? PF_OK : PF_ERR_TIMEOUT;
+}
+
+size_t pf_lowrank_linear_workspace(int64_t m, int64_t k, int64_t n, int64_t r, int dtype, int is_bwd) {
+    if (!valid_dtype(dtype) || m < 0 || k < 1 || n < 1 || r < 1) return 0;
+    return linear_ws(m, k, n, r, dtype, is_bwd != 0).total;
+}
+
+int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
+                          int64_t ldv, void* y, int64_t ldy, void* T_stash, int64_t ldt,
+                          int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    int st = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
+    if (st != PF_OK) return st;
+    if (!y || ldy < n || !elem_aligned(y, dtype)) return PF_ERR_INVALID_ARG;
+    if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
+    const LinearWs w = linear_ws(m, k, n, r, dtype, false);
+    st = check_ws(workspace, workspace_bytes, w.total);
+    if (st != PF_OK) return st;
+    if (m == 0) return PF_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+
+    if (dtype == PF_BF16) {
+        tc::LinearArgs a;
+        a.x = x; a.ldx = ldx; a.U = U; a.ldu = ldu; a.V = V; a.ldv = ldv;
+        a.y = y; a.ldy = ldy; a.T = T_stash; a.ldt = ldt;
+        a.m = m; a.k = k; a.n = n; a.r = r;
+        a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.stream = stream;
+        int handled = 0;
+        st = tc::linear_fwd(a, &handled);
+        if (st != PF_OK || handled) return st;
+    }
+    void* T = T_stash ? T_stash : static_cast<void*>(ws + w.off_T);
+    const int64_t ldT = T_stash ? ldt : r;
+    PF_CUDA(simt_gemm(mk(plainA(x, ldx, 1), plainB(U, ldu, 1), T, ldT, m, r, k, dtype), stream));
+    PF_CUDA(simt_gemm(mk(plainA(T, ldT, 1), plainB(V, 1, ldv), y, ldy, m, n, r, dtype), stream));
+    return PF_OK;
+}
+
+int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
+                          int64_t ldv, const void* dY, int64_t lddy, const void* T_stash, int64_t ldt,
+                          void* dX, int64_t lddx, void* dU, int64_t lddu, void* dV, int64_t lddv,
+                          int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    int st = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
+    if (st != PF_OK) return st;
+    if (!dY || lddy < n || !elem_aligned(dY, dtype)) return PF_ERR_INVALID_ARG;
+    if (!dU || lddu < r || !elem_aligned(dU, dtype)) return PF_ERR_INVALID_ARG;
+    if (!dV || lddv < r || !elem_aligned(dV, dtype)) return PF_ERR_INVALID_ARG;
+    if (dX && (lddx < k || !elem_aligned(dX, dtype))) return PF_ERR_INVALID_ARG;
+    if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
+    const LinearWs w = linear_ws(m, k, n, r, dtype, true);
+    st = check_ws(workspace, workspace_bytes, w.total);
+    if (st != PF_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t s = dtype_size(dtype);
+    if (m == 0) {  // empty sums
+        PF_CUDA(cudaMemset2DAsync(dU, lddu * s, 0, r * s, k, stream));
+        PF_CUDA(cudaMemset2DAsync(dV, lddv * s, 0, r * s, n, stream));
+        return PF_OK;
+    }
+    char* ws = static_cast<char*>(workspace);
+
+    if (dtype == PF_BF16) {
+        tc::LinearArgs a;
+        a.x = x; a.ldx = ldx; a.U = U; a.ldu = ldu; a.V = V; a.ldv = ldv;
+        a.dY = dY; a.lddy = lddy; a.T = const_cast<void*>(T_stash); a.ldt = ldt;
+        a.dX = dX; a.lddx = lddx; a.dU = dU; a.lddu = lddu; a.dV = dV; a.lddv = lddv;
+        a.m = m; a.k = k; a.n = n; a.r = r;
+        a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.ws_G = ws + w.off_G; a.stream = stream;
+        int handled = 0;
+        st = tc::linear_bwd(a, &handled);
+        if (st != PF_OK || handled) return st;
+    }
+    const void* T = T_stash;
+    int64_t ldT = ldt;
+    if (!T) {
+        void* Tw = ws + w.off_T;
+        PF_CUDA(simt_gemm(mk(plainA(x, ldx, 1), plainB(U, ldu, 1), Tw, r, m, r, k, dtype), stream));
+        T = Tw; ldT = r;
+    }
+    void* G = ws + w.off_G;
+    float* partial = reinterpret_cast<float*>(ws + w.off_partial);
+    PF_CUDA(simt_gemm(mk(plainA(dY, lddy, 1), plainB(V, ldv, 1), G, r, m, r, n, dtype), stream));
+    if (dX) PF_CUDA(simt_gemm(mk(plainA(G, r, 1), plainB(U, 1, ldu), dX, lddx, m, k, r, dtype), stream));
+    PF_CUDA(simt_gemm(mk(plainA(x, 1, ldx), plainB(G, r, 1), dU, lddu, k, r, m, dtype, w.splits_dU, partial), stream));
+    PF_CUDA(simt_gemm(mk(plainA(dY, 1, lddy), plainB(T, ldT, 1), dV, lddv, n, r, m, dtype, w.splits_dV, partial), stream));
+    return PF_OK;
+}
+
+// ------------------------------------------------------------------------------ conv
+namespace {
+struct ConvWs {
+    size_t off_T, off_dT, off_partial, off_tc, total;
+    int splits_dU, splits_dV;
+    int Ho, Wo;
+    int64_t P, Pin;
+};
+ConvWs conv_ws(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride, int pad,
+               int dtype, bool bwd) {
+    ConvWs w;
+    std::memset(&w, 0, sizeof(w));
+    w.Ho = (H + 2 * pad - kh) / stride + 1;
+    w.Wo = (W + 2 * pad - kw) / stride + 1;
+    if (w.Ho < 0) w.Ho = 0;
+    if (w.Wo < 0) w.Wo = 0;
+    w.P = static_cast<int64_t>(N) * w.Ho * w.Wo;
+    w.Pin = static_cast<int64_t>(N) * H * W;
+    const size_t s = dtype_size(dtype);
+    size_t off = 0;
+    w.off_T = off; off += align_up(static_cast<size_t>(w.P) * R * s, 256);
+    if (bwd) {
+        w.off_dT = off; off += align_up(static_cast<size_t>(w.P) * R * s, 256);
+        const int64_t Keff = static_cast<int64_t>(kh) * kw * C;
+        w.splits_dU = simt_pick_splits(Keff, R, w.P);
+        w.splits_dV = simt_pick_splits(O, R, w.P);
+        size_t pu = w.splits_dU > 1 ? static_cast<size_t>(w.splits_dU) * Keff * R * 4 : 0;
+        size_t pv = w.splits_dV > 1 ? static_cast<size_t>(w.splits_dV) * O * R * 4 : 0;
+        w.off_partial = off; off += align_up(pu > pv ? pu : pv, 256);
+    }
+    w.off_tc = off;
+    if (dtype == PF_BF16) off += align_up(tc::conv_extra_workspace(N, H, W, C, R, O, kh, kw, stride, pad, bwd), 256);
+    w.total = off;
+    return w;
+}
+int validate_conv_common(const void* x, const void* U, const void* V, int N, int H, int W, int C,
+                         int R, int O, int kh, int kw, int stride, int pad, int dtype) {
+    if (!valid_dtype(dtype)) return PF_ERR_INVALID_ARG;
+    if (N < 0 || H < 1 || W < 1 || C < 1 || R < 1 || O < 1 || kh < 1 || kw < 1 || pad < 0)
+        return PF_ERR_INVALID_ARG;
+    if (stride < 1 || kh != kw) return PF_ERR_UNSUPPORTED;
+    if (H + 2 * pad < kh || W + 2 * pad < kw) return PF_ERR_INVALID_ARG;
+    if (!x || !U || !V) return PF_ERR_INVALID_ARG;
+    if (!elem_aligned(x, dtype) || !elem_aligned(U, dtype) || !elem_aligned(V, dtype))
+        return PF_ERR_INVALID_ARG;
+    return PF_OK;
+}
+ConvGeom geom(int N, int H, int W, int C, int R, int kh, int kw, int stride, int pad, const ConvWs& w) {
+    ConvGeom g;
+    g.N = N; g.H = H; g.W = W; g.C = C; g.Ho = w.Ho; g.Wo = w.Wo; g.kh = kh; g.kw = kw;
+    g.st = stride; g.pad = pad; g.R = R;
+    return g;
+}
+}  // namespace
+
+size_t pf_lowrank_conv_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw,
+                                 int stride, int pad, int dtype, int is_bwd) {
+    if (!valid_dtype(dtype) || N < 0 || H < 1 || W < 1 || C < 1 || R < 1 || O < 1 || kh < 1 ||
+        kw < 1 || pad < 0 || stride < 1 || H + 2 * pad < kh || W + 2 * pad < kw)
+        return 0;
+    return conv_ws(N, H, W, C, R, O, kh, kw, stride, pad, dtype, is_bwd != 0).total;
+}
+
+int pf_lowrank_conv_fwd(const void* x, const void* U, const void* V, void* y, void* T_stash,
+                        int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
+                        int pad, int dtype, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    int st = validate_conv_common(x, U, V, N, H, W, C, R, O, kh, kw, stride, pad, dtype);
+    if (st != PF_OK) return st;
+    if (!y || !elem_aligned(y, dtype) || (T_stash && !elem_aligned(T_stash, dtype)))
+        return PF_ERR_INVALID_ARG;
+    const ConvWs w = conv_ws(N, H, W, C, R, O, kh, kw, stride, pad, dtype, false);
+    st = check_ws(workspace, workspace_bytes, w.total);
+    if (st != PF_OK) return st;
+    if (w.P == 0) return PF_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+
+    if (dtype == PF_BF16) {
+        tc::ConvArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.x = x; a.U = U; a.V = V; a.y = y; a.T = T_stash;
+        a.N = N; a.H = H; a.W = W; a.C = C; a.R = R; a.O = O; a.kh = kh; a.kw = kw;
+        a.stride = stride; a.pad = pad; a.Ho = w.Ho; a.Wo = w.Wo;
+        a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.stream = stream;
+        int handled = 0;
+        st = tc::conv_fwd(a, &handled);
+        if (st != PF_OK || handled) return st;
+    }
+    void* T = T_stash ? T_stash : static_cast<void*>(ws + w.off_T);
+    MatA A;
+    std::memset(&A, 0, sizeof(A));
+    A.p = x; A.kind = A_IM2COL; A.l_fast = 1; A.g = geom(N, H, W, C, R, kh, kw, stride, pad, w);
+    const int64_t Keff = static_cast<int64_t>(kh) * kw * C;
+    PF_CUDA(simt_gemm(mk(A, plainB(U, R, 1), T, R, w.P, R, Keff, dtype), stream));
+    PF_CUDA(simt_gemm(mk(plainA(T, R, 1), plainB(V, 1, R), y, O, w.P, O, R, dtype), stream));
+    return PF_OK;
+}
+
+int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void* dY,
+                        const void* T_stash, void* dX, void* dU, void* dV,
+                        int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
+                        int pad, int dtype, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    int st = validate_conv_common(x, U, V, N, H, W, C, R, O, kh, kw, stride, pad, dtype);
+    if (st != PF_OK) return st;
+    if (!dY || !dU || !dV) return PF_ERR_INVALID_ARG;
+    if (!elem_aligned(dY, dtype) || !elem_aligned(dU, dtype) || !elem_aligned(dV, dtype) ||
+        (dX && !elem_aligned(dX, dtype)) || (T_stash && !elem_aligned(T_stash, dtype)))
+        return PF_ERR_INVALID_ARG;
+    const ConvWs w = conv_ws(N, H, W, C, R, O, kh, kw, stride, pad, dtype, true);
+    st = check_ws(workspace, workspace_bytes, w.total);
+    if (st != PF_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t s = dtype_size(dtype);
+    const int64_t Keff = static_cast<int64_t>(kh) * kw * C;
+    if (w.P == 0) {
+        PF_CUDA(cudaMemsetAsync(dU, 0, Keff * R * s, stream));
+        PF_CUDA(cudaMemsetAsync(dV, 0, static_cast<size_t>(O) * R * s, stream));
+        if (dX && w.Pin > 0) PF_CUDA(cudaMemsetAsync(dX, 0, w.Pin * C * s, stream));
+        return PF_OK;
+    }
+    char* ws = static_cast<char*>(workspace);
+
+    if (dtype == PF_BF16) {
+        tc::ConvArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.x = x; a.U = U; a.V = V; a.dY = dY; a.T = const_cast<void*>(T_stash);
+        a.dX = dX; a.dU = dU; a.dV = dV;
+        a.N = N; a.H = H; a.W = W; a.C = C; a.R = R; a.O = O; a.kh = kh; a.kw = kw;
+        a.stride = stride; a.pad = pad; a.Ho = w.Ho; a.Wo = w.Wo;
+        a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.ws_G = ws + w.off_dT; a.stream = stream;
+        int handled = 0;
+        st = tc::conv_bwd(a, &handled);
+        if (st != PF_OK || handled) return st;
+    }
+    MatA Aim;
+    std::memset(&Aim, 0, sizeof(Aim));
+    Aim.p = x; Aim.kind = A_IM2COL; Aim.l_fast = 1; Aim.g = geom(N, H, W, C, R, kh, kw, stride, pad, w);
+    const void* T = T_stash;
+    if (!T) {
+        void* Tw = ws + w.off_T;
+        PF_CUDA(simt_gemm(mk(Aim, plainB(U, R, 1), Tw, R, w.P, R, Keff, dtype), stream));
+        T = Tw;
+    }
+    void* dT = ws + w.off_dT;
+    float* partial = reinterpret_cast<float*>(ws + w.off_partial);
+    PF_CUDA(simt_gemm(mk(plainA(dY, O, 1), plainB(V, R, 1), dT, R, w.P, R, O, dtype), stream));
+    PF_CUDA(simt_gemm(mk(plainA(dY, 1, O), plainB(T, R, 1), dV, R, O, R, w.P, dtype, w.splits_dV, partial), stream));
+    MatA At = Aim;
+    At.kind = A_IM2COL_T; At.l_fast = 0;
+    PF_CUDA(simt_gemm(mk(At, plainB(dT, R, 1), dU, R, Keff, R, w.P, dtype, w.splits_dU, partial), stream));
+    if (dX) {
+        MatA Ac = Aim;
+        Ac.p = dT; Ac.kind = A_COL2IM; Ac.l_fast = 1;
+        MatB Bt;
+        std::memset(&Bt, 0, sizeof(Bt));
+        Bt.p = U; Bt.kind = B_TAPSPLIT; Bt.l_fast = 1; Bt.R = R; Bt.CR = C * R;
+        PF_CUDA(simt_gemm(mk(Ac, Bt, dX, C, w.Pin, C, static_cast<int64_t>(kh) * kw * R, dtype), stream));
+    }
+    return PF_OK;
+}
+
+// ------------------------------------------------------------------------------ pack
+int pf_pack_factor_grads(const void* const* grads, const int64_t* numels, int count, int dtype,
+                         void* flat, int64_t flat_capacity_elems, int64_t* offsets_out,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    (void)workspace; (void)workspace_bytes;
+    if (!valid_dtype(dtype) || count < 0 || !offsets_out || flat_capacity_elems < 0)
+        return PF_ERR_INVALID_ARG;
+    if (count > 0 && (!grads || !numels)) return PF_ERR_INVALID_ARG;
+    offsets_out[0] = 0;
+    for (int i = 0; i < count; ++i) {
+        if (numels[i] < 0) return PF_ERR_INVALID_ARG;
+        if (numels[i] > 0 && (!grads[i] || !elem_aligned(grads[i], dtype))) return PF_ERR_INVALID_ARG;
+        if (numels[i] > (1LL << 46)) return PF_ERR_UNSUPPORTED;
+        offsets_out[i + 1] = offsets_out[i] + numels[i];
+    }
+    const int64_t total = offsets_out[count];
+    if (total > flat_capacity_elems) return PF_ERR_WORKSPACE;
+    if (total == 0) return PF_OK;
+    if (!flat || !elem_aligned(flat, dtype)) return PF_ERR_INVALID_ARG;
+    PF_CUDA(pack_launch(grads, numels, offsets_out, count, static_cast<int>(dtype_size(dtype)), flat,
+                        static_cast<cudaStream_t>(cuda_stream)));
+    return PF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,83 @@
+// Internal declarations shared by the translation units of libpf (not part of the ABI).
+#ifndef PF_INTERNAL_H_
+#define PF_INTERNAL_H_
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "pf.h"
+
+namespace pf {
+
+constexpr int kNumSMs = 148;  // B200
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t dtype_size(int dtype) { return dtype == PF_BF16 ? 2 : 4; }
+
+// ---------------------------------------------------------------------------------------
+// Generic strided / implicit matrix views consumed by the FMA (SIMT) GEMM.  The FMA path
+// serves fp32 storage and every bf16 shape outside the tensor-core envelope.
+// ---------------------------------------------------------------------------------------
+enum AKind : int {
+    A_PLAIN = 0,     // A(i,l) = p[i*s_row + l*s_col]
+    A_IM2COL = 1,    // i = output pixel (n,ho,wo), l = (a,b,c):  x[n, ho*st-pad+a, wo*st-pad+b, c] or 0
+    A_IM2COL_T = 2,  // i = (a,b,c), l = output pixel: same value, roles swapped (for dU)
+    A_COL2IM = 3     // i = input pixel (n,h,w), l = (a,b,j): dT[n,(h+pad-a)/st,(w+pad-b)/st,j] or 0
+};
+enum BKind : int {
+    B_PLAIN = 0,    // B(l,j) = p[l*s_row + j*s_col]
+    B_TAPSPLIT = 1  // l = (tap, q), q < R:  p[tap*C*R + j*R + q]   (U[tap][j][q] read as (tap,q) x j)
+};
+
+struct ConvGeom {
+    int N, H, W, C, Ho, Wo, kh, kw, st, pad, R;
+};
+
+struct MatA {
+    const void* p;
+    int64_t s_row, s_col;
+    int kind;
+    int l_fast;  // 1 if consecutive l are contiguous in memory, else consecutive i are
+    ConvGeom g;
+};
+struct MatB {
+    const void* p;
+    int64_t s_row, s_col;
+    int kind;
+    int l_fast;
+    int R, CR;  // B_TAPSPLIT only
+};
+
+struct SimtGemm {
+    MatA A;
+    MatB B;
+    void* C;          // [M, N] row-major, ldc, storage dtype
+    int64_t ldc;
+    int64_t M, N, K;
+    int splits;       // > 1: fp32 partials go to `partial` [splits, M, N], then a fixed-order sum
+    float* partial;
+    int dtype;
+};
+
+cudaError_t simt_gemm(const SimtGemm& g, cudaStream_t stream);
+int simt_pick_splits(int64_t M, int64_t N, int64_t K);
+
+// Strided 2-D copy with zero fill (repack to a padded pitch), elements of 2 bytes.
+cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t ld_dst,
+                             int64_t rows, int64_t cols, int64_t cols_padded, cudaStream_t stream);
+
+// pack
+cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const int64_t* offsets,
+                        int count, int elem_bytes, void* flat, cudaStream_t stream);
+
+// host-side count of kernels launched by this library
+void count_launch(int n = 1);
+
+// device status word (bounded waits report here)
+cudaError_t read_and_clear_device_status(unsigned int* out);
+
+}  // namespace pf
+#endif

@@ -1,0 +1,223 @@
+// FMA (CUDA-core) GEMM with implicit-matrix views.
+//
+// Serves the fp32 storage path (single-pass TF32 cannot reach 1e-4 after two chained
+// products) and every bf16 shape outside the tensor-core envelope.  One kernel, templated on
+// how operand A is addressed: plain strided, im2col of an NHWC image (convolution forward
+// and dU), or the gather form of the transposed convolution (dX).  Products accumulate in
+// fp32; a reduction split over K writes fp32 partials that a second kernel sums in a fixed
+// order, so results are bit-reproducible run to run.
+#include "pf_internal.h"
+
+namespace pf {
+namespace {
+
+constexpr int BM = 64, BN = 64, BK = 16, NT = 256;
+
+template <typename T> __device__ __forceinline__ float ldf(const void* p, int64_t idx);
+template <> __device__ __forceinline__ float ldf<float>(const void* p, int64_t idx) {
+    return __ldg(reinterpret_cast<const float*>(p) + idx);
+}
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const void* p, int64_t idx) {
+    const unsigned short raw = __ldg(reinterpret_cast<const unsigned short*>(p) + idx);
+    return __uint_as_float(static_cast<unsigned int>(raw) << 16);
+}
+template <typename T> __device__ __forceinline__ void stf(void* p, int64_t idx, float v);
+template <> __device__ __forceinline__ void stf<float>(void* p, int64_t idx, float v) {
+    reinterpret_cast<float*>(p)[idx] = v;
+}
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(void* p, int64_t idx, float v) {
+    reinterpret_cast<__nv_bfloat16*>(p)[idx] = __float2bfloat16_rn(v);
+}
+
+template <typename T, int AK>
+__device__ __forceinline__ float load_a(const MatA& A, int64_t i, int64_t l) {
+    if (AK == A_PLAIN) {
+        return ldf<T>(A.p, i * A.s_row + l * A.s_col);
+    } else if (AK == A_IM2COL || AK == A_IM2COL_T) {
+        const int64_t pix = (AK == A_IM2COL) ? i : l;
+        const int64_t q = (AK == A_IM2COL) ? l : i;
+        const ConvGeom& g = A.g;
+        const int c = static_cast<int>(q % g.C);
+        const int tap = static_cast<int>(q / g.C);
+        const int b = tap % g.kw, a = tap / g.kw;
+        const int wo = static_cast<int>(pix % g.Wo);
+        const int64_t t = pix / g.Wo;
+        const int ho = static_cast<int>(t % g.Ho);
+        const int64_t n = t / g.Ho;
+        const int h = ho * g.st - g.pad + a, w = wo * g.st - g.pad + b;
+        if (h < 0 || h >= g.H || w < 0 || w >= g.W) return 0.f;
+        return ldf<T>(A.p, ((n * g.H + h) * g.W + w) * g.C + c);
+    } else {  // A_COL2IM
+        const ConvGeom& g = A.g;
+        const int j = static_cast<int>(l % g.R);
+        const int tap = static_cast<int>(l / g.R);
+        const int b = tap % g.kw, a = tap / g.kw;
+        const int w = static_cast<int>(i % g.W);
+        const int64_t t = i / g.W;
+        const int h = static_cast<int>(t % g.H);
+        const int64_t n = t / g.H;
+        const int hn = h + g.pad - a, wn = w + g.pad - b;
+        if (hn < 0 || wn < 0 || hn % g.st != 0 || wn % g.st != 0) return 0.f;
+        const int ho = hn / g.st, wo = wn / g.st;
+        if (ho >= g.Ho || wo >= g.Wo) return 0.f;
+        return ldf<T>(A.p, ((n * g.Ho + ho) * g.Wo + wo) * g.R + j);
+    }
+}
+
+template <typename T, int BKD>
+__device__ __forceinline__ float load_b(const MatB& B, int64_t l, int64_t j) {
+    if (BKD == B_PLAIN) return ldf<T>(B.p, l * B.s_row + j * B.s_col);
+    const int64_t tap = l / B.R, q = l % B.R;
+    return ldf<T>(B.p, tap * B.CR + j * B.R + q);
+}
+
+template <typename T, int AK, int BKD>
+__global__ void __launch_bounds__(NT)
+simt_gemm_kernel(const SimtGemm g) {
+    __shared__ float As[BK][BM + 1];
+    __shared__ float Bs[BK][BN + 1];
+    const int tid = threadIdx.x;
+    const int tx = tid % 16, ty = tid / 16;
+    const int64_t i0 = static_cast<int64_t>(blockIdx.x) * BM;
+    const int64_t j0 = static_cast<int64_t>(blockIdx.y) * BN;
+    const int64_t kchunk = (g.K + g.splits - 1) / g.splits;
+    const int64_t kbeg = static_cast<int64_t>(blockIdx.z) * kchunk;
+    const int64_t kend = kbeg + kchunk < g.K ? kbeg + kchunk : g.K;
+
+    float acc[4][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = 0.f;
+
+    for (int64_t l0 = kbeg; l0 < kend; l0 += BK) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int li, ii;
+            if (g.A.l_fast) { li = tid % BK; ii = tid / BK + (NT / BK) * q; }
+            else            { ii = tid % BM; li = tid / BM + (NT / BM) * q; }
+            const int64_t gi = i0 + ii, gl = l0 + li;
+            As[li][ii] = (gi < g.M && gl < kend) ? load_a<T, AK>(g.A, gi, gl) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int li, ji;
+            if (g.B.l_fast) { li = tid % BK; ji = tid / BK + (NT / BK) * q; }
+            else            { ji = tid % BN; li = tid / BN + (NT / BN) * q; }
+            const int64_t gj = j0 + ji, gl = l0 + li;
+            Bs[li][ji] = (gj < g.N && gl < kend) ? load_b<T, BKD>(g.B, gl, gj) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int l = 0; l < BK; ++l) {
+            float a[4], b[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) a[u] = As[l][ty * 4 + u];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) b[v] = Bs[l][tx * 4 + v];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(a[u], b[v], acc[u][v]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int64_t gi = i0 + ty * 4 + u;
+        if (gi >= g.M) continue;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int64_t gj = j0 + tx * 4 + v;
+            if (gj >= g.N) continue;
+            if (g.splits > 1) g.partial[(static_cast<int64_t>(blockIdx.z) * g.M + gi) * g.N + gj] = acc[u][v];
+            else stf<T>(g.C, gi * g.ldc + gj, acc[u][v]);
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ partial, void* C, int64_t ldc, int64_t M, int64_t N,
+                     int splits) {
+    const int64_t total = M * N;
+    for (int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
+         e += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        float s = 0.f;
+        for (int z = 0; z < splits; ++z) s += partial[static_cast<int64_t>(z) * total + e];
+        stf<T>(C, (e / N) * ldc + (e % N), s);
+    }
+}
+
+template <typename T>
+cudaError_t launch_typed(const SimtGemm& g, cudaStream_t stream) {
+    dim3 grid(static_cast<unsigned>(ceil_div(g.M, BM)), static_cast<unsigned>(ceil_div(g.N, BN)),
+              static_cast<unsigned>(g.splits));
+    if (g.A.kind == A_PLAIN && g.B.kind == B_PLAIN)
+        simt_gemm_kernel<T, A_PLAIN, B_PLAIN><<<grid, NT, 0, stream>>>(g);
+    else if (g.A.kind == A_IM2COL && g.B.kind == B_PLAIN)
+        simt_gemm_kernel<T, A_IM2COL, B_PLAIN><<<grid, NT, 0, stream>>>(g);
+    else if (g.A.kind == A_IM2COL_T && g.B.kind == B_PLAIN)
+        simt_gemm_kernel<T, A_IM2COL_T, B_PLAIN><<<grid, NT, 0, stream>>>(g);
+    else if (g.A.kind == A_COL2IM && g.B.kind == B_TAPSPLIT)
+        simt_gemm_kernel<T, A_COL2IM, B_TAPSPLIT><<<grid, NT, 0, stream>>>(g);
+    else
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    count_launch();
+    if (g.splits > 1) {
+        const int64_t total = g.M * g.N;
+        const int blocks = static_cast<int>(ceil_div(total, 256) < 4 * kNumSMs ? ceil_div(total, 256)
+                                                                                : 4 * kNumSMs);
+        splitk_reduce_kernel<T><<<blocks, 256, 0, stream>>>(g.partial, g.C, g.ldc, g.M, g.N, g.splits);
+        e = cudaGetLastError();
+        if (e == cudaSuccess) count_launch();
+    }
+    return e;
+}
+
+__global__ void __launch_bounds__(256)
+repack_rows_kernel(const unsigned short* __restrict__ src, int64_t ld_src,
+                   unsigned short* __restrict__ dst, int64_t ld_dst, int64_t rows, int64_t cols,
+                   int64_t cols_padded) {
+    const int64_t total = rows * cols_padded;
+    for (int64_t e = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
+         e += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t rr = e / cols_padded, cc = e % cols_padded;
+        dst[rr * ld_dst + cc] = cc < cols ? src[rr * ld_src + cc] : static_cast<unsigned short>(0);
+    }
+}
+
+}  // namespace
+
+int simt_pick_splits(int64_t M, int64_t N, int64_t K) {
+    const int64_t tiles = ceil_div(M, BM) * ceil_div(N, BN);
+    int64_t s = ceil_div(2 * kNumSMs, tiles);
+    const int64_t max_by_k = ceil_div(K, 8 * BK);
+    if (s > max_by_k) s = max_by_k;
+    if (s > 64) s = 64;
+    if (s < 1) s = 1;
+    return static_cast<int>(s);
+}
+
+cudaError_t simt_gemm(const SimtGemm& g, cudaStream_t stream) {
+    if (g.M <= 0 || g.N <= 0) return cudaSuccess;
+    if (ceil_div(g.N, BN) > 65535 || ceil_div(g.M, BM) > 2147483647LL) return cudaErrorInvalidConfiguration;
+    return g.dtype == PF_BF16 ? launch_typed<__nv_bfloat16>(g, stream) : launch_typed<float>(g, stream);
+}
+
+cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t ld_dst,
+                             int64_t rows, int64_t cols, int64_t cols_padded, cudaStream_t stream) {
+    const int64_t total = rows * cols_padded;
+    if (total <= 0) return cudaSuccess;
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 8 * kNumSMs ? ceil_div(total, 256)
+                                                                            : 8 * kNumSMs);
+    repack_rows_kernel<<<blocks, 256, 0, stream>>>(static_cast<const unsigned short*>(src), ld_src,
+                                                   static_cast<unsigned short*>(dst), ld_dst, rows, cols,
+                                                   cols_padded);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace pf

@@ -1,0 +1,42 @@
+// Tensor-core (tcgen05 / TMEM / TMA) path for bf16 storage.  Each entry either handles the
+// call (*handled = 1) or declines it (*handled = 0, nothing launched) when the shape lies
+// outside its envelope; the caller then uses the FMA kernels.
+#ifndef PF_TC_H_
+#define PF_TC_H_
+
+#include "pf_internal.h"
+
+namespace pf {
+
+unsigned int* device_status_ptr();  // per-device address of the bounded-wait status word
+
+namespace tc {
+
+struct LinearArgs {
+    const void *x = nullptr, *U = nullptr, *V = nullptr, *dY = nullptr;
+    void *y = nullptr, *T = nullptr, *dX = nullptr, *dU = nullptr, *dV = nullptr;
+    int64_t ldx = 0, ldu = 0, ldv = 0, ldy = 0, ldt = 0, lddy = 0, lddx = 0, lddu = 0, lddv = 0;
+    int64_t m = 0, k = 0, n = 0, r = 0;
+    char *ws = nullptr, *ws_T = nullptr, *ws_G = nullptr;
+    cudaStream_t stream = nullptr;
+};
+
+struct ConvArgs {
+    const void *x, *U, *V, *dY;
+    void *y, *T, *dX, *dU, *dV;
+    int N, H, W, C, R, O, kh, kw, stride, pad, Ho, Wo;
+    char *ws, *ws_T, *ws_G;
+    cudaStream_t stream;
+};
+
+size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool bwd);
+size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
+                            int pad, bool bwd);
+int linear_fwd(const LinearArgs& a, int* handled);
+int linear_bwd(const LinearArgs& a, int* handled);
+int conv_fwd(const ConvArgs& a, int* handled);
+int conv_bwd(const ConvArgs& a, int* handled);
+
+}  // namespace tc
+}  // namespace pf
+#endif

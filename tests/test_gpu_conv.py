@@ -1,0 +1,109 @@
+"""GPU parity: factorized NHWC convolution forward/backward through the C ABI vs the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2103_03936_b200 as pf
+import pf_workloads as wl
+from _gpu import Guarded, assert_close, dev
+
+pytestmark = pytest.mark.gpu
+
+
+def run_conv(case, stash=True, need_dX=True):
+    d = case.generate()
+    dt = case.dtype
+    x, U, V, dY = (dev(d[k_], dt) for k_ in ("x", "U", "V", "dY"))
+    Ho, Wo = case.Ho, case.Wo
+    gy = Guarded((case.N, Ho, Wo, case.O), dt)
+    gT = Guarded((case.N, Ho, Wo, case.R), dt)
+    pf.pf_lowrank_conv_fwd(x, U, V, stride=case.stride, pad=case.pad, y=gy.t,
+                           T_stash=gT.t if stash else None)
+    gdX, gdU, gdV = Guarded(x.shape, dt), Guarded(U.shape, dt), Guarded(V.shape, dt)
+    pf.pf_lowrank_conv_bwd(x, U, V, dY, stride=case.stride, pad=case.pad,
+                           T_stash=gT.t if stash else None, need_dX=need_dX,
+                           dX=gdX.t if need_dX else None, dU=gdU.t, dV=gdV.t)
+    torch.cuda.synchronize()
+    y_ref, T_ref = oracle.conv_fwd(d["x"], d["U"], d["V"], case.stride, case.pad)
+    dX_ref, dU_ref, dV_ref = oracle.conv_bwd(d["x"], d["U"], d["V"], d["dY"], case.stride, case.pad)
+    errs = {"y": assert_close(gy.t, y_ref, dt, "y")}
+    if stash:
+        errs["T"] = assert_close(gT.t, T_ref, dt, "T")
+    if need_dX:
+        errs["dX"] = assert_close(gdX.t, dX_ref, dt, "dX")
+    errs["dU"] = assert_close(gdU.t, dU_ref, dt, "dU")
+    errs["dV"] = assert_close(gdV.t, dV_ref, dt, "dV")
+    for g in (gy, gT, gdX, gdU, gdV):
+        g.check()
+    assert pf.pf_last_device_status() == 0
+    return errs
+
+
+SMALL = [  # N,H,W,C,R,O,k,stride,pad
+    (1, 1, 1, 1, 1, 1, 1, 1, 0),
+    (1, 3, 3, 1, 1, 1, 3, 1, 1),
+    (2, 5, 4, 3, 2, 3, 3, 1, 1),
+    (1, 6, 5, 2, 3, 2, 3, 2, 1),
+    (2, 4, 4, 2, 2, 3, 1, 1, 0),
+    (1, 5, 5, 2, 2, 2, 3, 1, 0),
+    (1, 7, 6, 2, 2, 2, 5, 2, 2),
+    (3, 9, 11, 8, 5, 16, 3, 1, 1),
+    (2, 8, 8, 16, 8, 24, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_small_shapes(dtype):
+    for i, (N, H, W, C, R, O, k, st, pad) in enumerate(SMALL):
+        run_conv(wl.ConvCase(f"s{i}", N, H, W, C, R, O, dtype, 50 + i, kh=k, kw=k, stride=st, pad=pad))
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+@pytest.mark.parametrize("N,H,W,C,R,O", [(2, 32, 32, 64, 16, 64), (3, 14, 14, 64, 16, 128),
+                                         (1, 20, 12, 72, 24, 40), (5, 16, 16, 128, 32, 128)])
+def test_multi_tile(dtype, N, H, W, C, R, O):
+    run_conv(wl.ConvCase("mt", N, H, W, C, R, O, dtype, 60))
+
+
+def test_recompute_without_stash_and_no_dX():
+    run_conv(wl.ConvCase("ns", 2, 16, 16, 64, 16, 64, wl.BF16, 61), stash=False)
+    run_conv(wl.ConvCase("nx", 2, 16, 16, 64, 16, 64, wl.BF16, 62), need_dX=False)
+
+
+@pytest.mark.parametrize("name,imgs", [("C4", [0, 63, 127]), ("C5b", [0, 100, 255])])
+def test_configs_full_size_sampled(name, imgs):
+    """Full-size conv configs: y, T, dX on sampled images (exact per image), dU, dV on sampled
+    rank columns (exact from column-sliced factors)."""
+    c = wl.conv_cases()[name]
+    d = c.generate()
+    x, U, V, dY = (dev(d[k_], c.dtype) for k_ in ("x", "U", "V", "dY"))
+    y, T = pf.pf_lowrank_conv_fwd(x, U, V, want_stash=True)
+    dX, dU, dV = pf.pf_lowrank_conv_bwd(x, U, V, dY, T_stash=T)
+    torch.cuda.synchronize()
+    y_ref, T_ref = oracle.conv_fwd(d["x"][imgs], d["U"], d["V"])
+    dX_ref, _, _ = oracle.conv_bwd(d["x"][imgs], d["U"], d["V"], d["dY"][imgs])
+    assert_close(y[imgs], y_ref, c.dtype, "y")
+    assert_close(T[imgs], T_ref, c.dtype, "T")
+    assert_close(dX[imgs], dX_ref, c.dtype, "dX")
+    J = [0, 31, 63]
+    _, dU_ref, dV_ref = oracle.conv_bwd(d["x"], d["U"][..., J], d["V"][:, J], d["dY"])
+    assert_close(dU[..., J], dU_ref, c.dtype, "dU")
+    assert_close(dV[:, J], dV_ref, c.dtype, "dV")
+    # the step ends with the flat gradient buffer of its factor gradients
+    flat, offs = pf.pf_pack_factor_grads([dU, dV])
+    torch.cuda.synchronize()
+    assert offs == [0, dU.numel(), dU.numel() + dV.numel()]
+    assert torch.equal(flat[:offs[1]], dU.reshape(-1)) and torch.equal(flat[offs[1]:], dV.reshape(-1))
+    assert pf.pf_last_device_status() == 0
+
+
+def test_empty_batch():
+    x = torch.empty((0, 8, 8, 8), dtype=torch.bfloat16, device="cuda")
+    U = torch.ones((3, 3, 8, 4), dtype=torch.bfloat16, device="cuda")
+    V = torch.ones((8, 4), dtype=torch.bfloat16, device="cuda")
+    y = pf.pf_lowrank_conv_fwd(x, U, V)
+    assert y.shape == (0, 8, 8, 8)
+    _, dU, dV = pf.pf_lowrank_conv_bwd(x, U, V, torch.empty((0, 8, 8, 8), dtype=torch.bfloat16, device="cuda"))
+    torch.cuda.synchronize()
+    assert torch.all(dU == 0) and torch.all(dV == 0)

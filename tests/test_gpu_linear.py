@@ -1,0 +1,178 @@
+"""GPU parity: factorized linear forward/backward through the C ABI vs the fp64 oracle."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2103_03936_b200 as pf
+import pf_workloads as wl
+from _gpu import Guarded, assert_close, dev, host
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(case, ld_pad=0, stash=True, need_dX=True):
+    d = case.generate()
+    dt = case.dtype
+    m, k, n, r = case.m, case.k, case.n, case.r
+
+    def up(a, cols):
+        if not ld_pad:
+            return dev(a, dt)
+        buf = torch.zeros((a.shape[0], cols + ld_pad), dtype=wl.to_torch(a[:1], dt).dtype, device="cuda")
+        buf[:, :cols] = dev(a, dt)
+        return buf[:, :cols]
+
+    x, U, V, dY = up(d["x"], k), up(d["U"], r), up(d["V"], r), up(d["dY"], n)
+    gy = Guarded((m, n), dt, ld=n + ld_pad if ld_pad else None)
+    gT = Guarded((m, r), dt, ld=r + ld_pad if ld_pad else None)
+    out = pf.pf_lowrank_linear_fwd(x, U, V, y=gy.t, T_stash=gT.t if stash else None)
+    y_ref, T_ref = oracle.linear_fwd(d["x"], d["U"], d["V"])
+    dX_ref, dU_ref, dV_ref = oracle.linear_bwd(d["x"], d["U"], d["V"], d["dY"])
+    gdX = Guarded((m, k), dt, ld=k + ld_pad if ld_pad else None)
+    gdU = Guarded((k, r), dt, ld=r + ld_pad if ld_pad else None)
+    gdV = Guarded((n, r), dt, ld=r + ld_pad if ld_pad else None)
+    pf.pf_lowrank_linear_bwd(x, U, V, dY, T_stash=gT.t if stash else None, need_dX=need_dX,
+                             dX=gdX.t if need_dX else None, dU=gdU.t, dV=gdV.t)
+    torch.cuda.synchronize()
+    errs = {"y": assert_close(gy.t, y_ref, dt, "y")}
+    if stash:
+        errs["T"] = assert_close(gT.t, T_ref, dt, "T")
+    if need_dX:
+        errs["dX"] = assert_close(gdX.t, dX_ref, dt, "dX")
+    errs["dU"] = assert_close(gdU.t, dU_ref, dt, "dU")
+    errs["dV"] = assert_close(gdV.t, dV_ref, dt, "dV")
+    for g in (gy, gT, gdX, gdU, gdV):
+        g.check()
+    assert pf.pf_last_device_status() == 0
+    return errs
+
+
+GRID = [(m, k, n, r) for m, k, n, r in itertools.product((1, 7, 130), (1, 17, 100), (3, 24, 130), (1, 5, 33))]
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_tiny_exhaustive_grid(dtype):
+    for idx, (m, k, n, r) in enumerate(GRID):
+        run_case(wl.LinearCase(f"g{idx}", m, k, n, r, dtype, 100 + idx))
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+@pytest.mark.parametrize("m,k,n,r", [(257, 72, 136, 24), (300, 200, 264, 40), (129, 64, 64, 64),
+                                     (1000, 328, 520, 96)])
+def test_multi_tile_ragged(dtype, m, k, n, r):
+    run_case(wl.LinearCase("rag", m, k, n, r, dtype, 7))
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_leading_dimensions_and_padding_untouched(dtype):
+    run_case(wl.LinearCase("ld", 200, 72, 136, 24, dtype, 8), ld_pad=8)
+    run_case(wl.LinearCase("ld", 77, 33, 50, 7, dtype, 9), ld_pad=3)
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_recompute_without_stash_and_no_dX(dtype):
+    run_case(wl.LinearCase("ns", 300, 136, 72, 24, dtype, 10), stash=False)
+    run_case(wl.LinearCase("nx", 300, 136, 72, 24, dtype, 11), need_dX=False)
+
+
+def test_config_C1_tiny_fp32():
+    run_case(wl.linear_cases()["C1"])
+
+
+@pytest.mark.parametrize("name", ["C2a", "C2b", "C3i", "C3h"])
+def test_configs_full_size(name):
+    errs = run_case(wl.linear_cases()[name])
+    print(name, errs)
+
+
+def test_config_C3_padded_pitch():
+    """LSTM shape with 16-byte-multiple row pitches (k 1500->1504, r 375->376 elements)."""
+    run_case(wl.linear_cases()["C3i"], ld_pad=0)
+    c = wl.linear_cases()["C3i"]
+    d = c.generate()
+
+    def padded(a, cols, ld):
+        buf = torch.zeros((a.shape[0], ld), dtype=torch.bfloat16, device="cuda")
+        buf[:, :cols] = dev(a, c.dtype)
+        return buf[:, :cols]
+    x, U, V, dY = padded(d["x"], 1500, 1504), padded(d["U"], 375, 376), padded(d["V"], 375, 376), dev(d["dY"], c.dtype)
+    y, T = pf.pf_lowrank_linear_fwd(x, U, V, want_stash=True)
+    dX, dU, dV = pf.pf_lowrank_linear_bwd(x, U, V, dY, T_stash=T)
+    y_ref, _ = oracle.linear_fwd(d["x"], d["U"], d["V"])
+    dX_ref, dU_ref, dV_ref = oracle.linear_bwd(d["x"], d["U"], d["V"], d["dY"])
+    for got, want, nm in ((y, y_ref, "y"), (dX, dX_ref, "dX"), (dU, dU_ref, "dU"), (dV, dV_ref, "dV")):
+        assert_close(got, want, c.dtype, nm)
+
+
+@pytest.fixture(scope="module")
+def sweep_inputs():
+    c = wl.linear_cases()["C5r16"]
+    x = wl.round_to(wl.normal(c.seed, 0, (c.m, c.k)), c.dtype)
+    dY = wl.round_to(wl.normal(c.seed, 3, (c.m, c.n)), c.dtype)
+    return x, dY, dev(x, c.dtype), dev(dY, c.dtype)
+
+
+@pytest.mark.parametrize("r", [16, 128, 256, 1024])
+def test_rank_sweep_full_size_sampled(sweep_inputs, r):
+    """m=16384, k=n=4096: y and dX on sampled rows, dU and dV on sampled rank columns (the
+    oracle computes those exactly from sliced inputs), in the configuration the bench times."""
+    x_h, dY_h, x, dY = sweep_inputs
+    c = wl.linear_cases()[f"C5r{r}"]
+    import math
+    sig = 1.0 / math.sqrt(c.k)
+    U_h = wl.round_to(wl.normal(c.factor_seed, 1, (c.k, r), sig), c.dtype)
+    V_h = wl.round_to(wl.normal(c.factor_seed, 2, (c.n, r), sig), c.dtype)
+    U, V = dev(U_h, c.dtype), dev(V_h, c.dtype)
+    y, T = pf.pf_lowrank_linear_fwd(x, U, V, want_stash=True)
+    dX, dU, dV = pf.pf_lowrank_linear_bwd(x, U, V, dY, T_stash=T)
+    torch.cuda.synchronize()
+    rows = [0, 1, 127, 128, 5000, 8191, 8192, 16383]
+    y_ref, T_ref = oracle.linear_fwd(x_h[rows], U_h, V_h)
+    dX_ref, _, _ = oracle.linear_bwd(x_h[rows], U_h, V_h, dY_h[rows])
+    assert_close(y[rows], y_ref, c.dtype, "y rows")
+    assert_close(T[rows], T_ref, c.dtype, "T rows")
+    assert_close(dX[rows], dX_ref, c.dtype, "dX rows")
+    J = sorted({0, r // 2, r - 1})
+    _, dU_ref, dV_ref = oracle.linear_bwd(x_h, U_h[:, J], V_h[:, J], dY_h)
+    assert_close(dU[:, J], dU_ref, c.dtype, "dU cols")
+    assert_close(dV[:, J], dV_ref, c.dtype, "dV cols")
+    assert pf.pf_last_device_status() == 0
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_backward_is_bit_reproducible(dtype):
+    c = wl.LinearCase("rep", 4096, 256, 320, 64, dtype, 12)
+    d = c.generate()
+    x, U, V, dY = (dev(d[k_], dtype) for k_ in ("x", "U", "V", "dY"))
+    a = pf.pf_lowrank_linear_bwd(x, U, V, dY)
+    b = pf.pf_lowrank_linear_bwd(x, U, V, dY)
+    torch.cuda.synchronize()
+    for p, q in zip(a, b):
+        assert torch.equal(p, q)
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_empty_batch(dtype):
+    tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
+    x = torch.empty((0, 16), dtype=tdt, device="cuda")
+    U = torch.ones((16, 4), dtype=tdt, device="cuda")
+    V = torch.ones((8, 4), dtype=tdt, device="cuda")
+    y = pf.pf_lowrank_linear_fwd(x, U, V)
+    assert y.shape == (0, 8)
+    dX, dU, dV = pf.pf_lowrank_linear_bwd(x, U, V, torch.empty((0, 8), dtype=tdt, device="cuda"),
+                                          dU=torch.full((16, 4), 3.0, dtype=tdt, device="cuda"),
+                                          dV=torch.full((8, 4), 3.0, dtype=tdt, device="cuda"))
+    torch.cuda.synchronize()
+    assert torch.all(dU == 0) and torch.all(dV == 0)
+
+
+def test_invalid_arguments_raise_not_launch():
+    x = torch.zeros((4, 8), dtype=torch.bfloat16, device="cuda")
+    U = torch.zeros((8, 2), dtype=torch.bfloat16, device="cuda")
+    V = torch.zeros((6, 2), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_lowrank_linear_fwd(x, U, V, workspace=torch.empty(8, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 3
