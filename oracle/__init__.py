@@ -70,7 +70,9 @@ def widen(a) -> np.ndarray:
     """Stored values -> float64, exactly.  uint16 arrays are bf16 bit patterns."""
     a = np.asarray(a)
     if a.dtype == np.uint16:
-        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+        a = np.ascontiguousarray(a)          # fancy-indexed slices may not be C-ordered
+        return np.ascontiguousarray((a.astype(np.uint32) << np.uint32(16)).view(np.float32),
+                                    dtype=np.float64)
     return np.ascontiguousarray(a, dtype=np.float64)
 
 

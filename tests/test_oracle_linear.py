@@ -124,3 +124,12 @@ def test_rel_err_metric():
     a = np.array([3.0, 4.0])
     assert oracle.rel_err(a, a) == 0.0
     assert abs(oracle.rel_err(a + np.array([0.3, 0.4]), a) - 0.1) < 1e-15
+
+
+def test_widen_returns_c_contiguous_for_sliced_bit_patterns():
+    """Column-sliced bf16 bit patterns (as used for sampled parity) must be marshalled in C order."""
+    import pf_workloads as wl
+    U = wl.round_to(np.arange(24, dtype=np.float64).reshape(2, 3, 4), wl.BF16)
+    w = oracle.widen(U[..., [0, 2]])
+    assert w.flags["C_CONTIGUOUS"]
+    np.testing.assert_array_equal(w, np.arange(24.0).reshape(2, 3, 4)[..., [0, 2]])
