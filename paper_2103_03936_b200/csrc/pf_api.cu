@@ -86,7 +86,7 @@ int validate_linear_common(const void* x, int64_t ldx, const void* U, int64_t ld
                            int64_t ldv, int64_t m, int64_t k, int64_t n, int64_t r, int dtype) {
     if (!valid_dtype(dtype)) return PF_ERR_INVALID_ARG;
     if (m < 0 || k < 1 || n < 1 || r < 1) return PF_ERR_INVALID_ARG;
-    if (!x || !U || !V) return PF_ERR_INVALID_ARG;
+    if ((!x && m > 0) || !U || !V) return PF_ERR_INVALID_ARG;   // an empty batch may be a null pointer
     if (ldx < k || ldu < r || ldv < r) return PF_ERR_INVALID_ARG;
     if (!elem_aligned(x, dtype) || !elem_aligned(U, dtype) || !elem_aligned(V, dtype))
         return PF_ERR_INVALID_ARG;
@@ -158,7 +158,7 @@ int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
     int st = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
     if (st != PF_OK) return st;
-    if (!y || ldy < n || !elem_aligned(y, dtype)) return PF_ERR_INVALID_ARG;
+    if ((!y && m > 0) || ldy < n || !elem_aligned(y, dtype)) return PF_ERR_INVALID_ARG;
     if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
     const LinearWs w = linear_ws(m, k, n, r, dtype, false);
     st = check_ws(workspace, workspace_bytes, w.total);
@@ -191,7 +191,7 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
     int st = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
     if (st != PF_OK) return st;
-    if (!dY || lddy < n || !elem_aligned(dY, dtype)) return PF_ERR_INVALID_ARG;
+    if ((!dY && m > 0) || lddy < n || !elem_aligned(dY, dtype)) return PF_ERR_INVALID_ARG;
     if (!dU || lddu < r || !elem_aligned(dU, dtype)) return PF_ERR_INVALID_ARG;
     if (!dV || lddv < r || !elem_aligned(dV, dtype)) return PF_ERR_INVALID_ARG;
     if (dX && (lddx < k || !elem_aligned(dX, dtype))) return PF_ERR_INVALID_ARG;
@@ -277,7 +277,7 @@ int validate_conv_common(const void* x, const void* U, const void* V, int N, int
         return PF_ERR_INVALID_ARG;
     if (stride < 1 || kh != kw) return PF_ERR_UNSUPPORTED;
     if (H + 2 * pad < kh || W + 2 * pad < kw) return PF_ERR_INVALID_ARG;
-    if (!x || !U || !V) return PF_ERR_INVALID_ARG;
+    if ((!x && N > 0) || !U || !V) return PF_ERR_INVALID_ARG;   // an empty batch may be a null pointer
     if (!elem_aligned(x, dtype) || !elem_aligned(U, dtype) || !elem_aligned(V, dtype))
         return PF_ERR_INVALID_ARG;
     return PF_OK;
@@ -304,7 +304,7 @@ int pf_lowrank_conv_fwd(const void* x, const void* U, const void* V, void* y, vo
                         void* cuda_stream) {
     int st = validate_conv_common(x, U, V, N, H, W, C, R, O, kh, kw, stride, pad, dtype);
     if (st != PF_OK) return st;
-    if (!y || !elem_aligned(y, dtype) || (T_stash && !elem_aligned(T_stash, dtype)))
+    if ((!y && N > 0) || !elem_aligned(y, dtype) || (T_stash && !elem_aligned(T_stash, dtype)))
         return PF_ERR_INVALID_ARG;
     const ConvWs w = conv_ws(N, H, W, C, R, O, kh, kw, stride, pad, dtype, false);
     st = check_ws(workspace, workspace_bytes, w.total);
@@ -341,7 +341,7 @@ int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void*
                         void* cuda_stream) {
     int st = validate_conv_common(x, U, V, N, H, W, C, R, O, kh, kw, stride, pad, dtype);
     if (st != PF_OK) return st;
-    if (!dY || !dU || !dV) return PF_ERR_INVALID_ARG;
+    if ((!dY && N > 0) || !dU || !dV) return PF_ERR_INVALID_ARG;
     if (!elem_aligned(dY, dtype) || !elem_aligned(dU, dtype) || !elem_aligned(dV, dtype) ||
         (dX && !elem_aligned(dX, dtype)) || (T_stash && !elem_aligned(T_stash, dtype)))
         return PF_ERR_INVALID_ARG;

@@ -64,6 +64,9 @@ struct SimtGemm {
 
 cudaError_t simt_gemm(const SimtGemm& g, cudaStream_t stream);
 int simt_pick_splits(int64_t M, int64_t N, int64_t K);
+// C[M,N] (storage dtype, ldc) = sum over z < splits of partial[z][M][N], in increasing z.
+cudaError_t splitk_reduce(const float* partial, void* C, int64_t ldc, int64_t M, int64_t N, int splits,
+                          int dtype, cudaStream_t stream);
 
 // Strided 2-D copy with zero fill (repack to a padded pitch), elements of 2 bytes.
 cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t ld_dst,

@@ -201,6 +201,18 @@ int simt_pick_splits(int64_t M, int64_t N, int64_t K) {
     return static_cast<int>(s);
 }
 
+cudaError_t splitk_reduce(const float* partial, void* C, int64_t ldc, int64_t M, int64_t N, int splits,
+                          int dtype, cudaStream_t stream) {
+    const int64_t total = M * N;
+    if (total <= 0) return cudaSuccess;
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 4 * kNumSMs ? ceil_div(total, 256) : 4 * kNumSMs);
+    if (dtype == PF_BF16) splitk_reduce_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(partial, C, ldc, M, N, splits);
+    else splitk_reduce_kernel<float><<<blocks, 256, 0, stream>>>(partial, C, ldc, M, N, splits);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
 cudaError_t simt_gemm(const SimtGemm& g, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
     if (ceil_div(g.N, BN) > 65535 || ceil_div(g.M, BM) > 2147483647LL) return cudaErrorInvalidConfiguration;

@@ -1,12 +1,426 @@
+// Tensor-core path (bf16 storage) for sm_100a: tcgen05 MMAs with accumulators in tensor memory,
+// operands staged in shared memory by TMA through an mbarrier pipeline.
+//
+// Kernel in this file:
+//   tc_gemm_kernel<BN>  C[M,N] = A * B for every operand orientation the factorized layers need
+//                       (row-major operands read either along or across the contraction index,
+//                       i.e. K-major or MN-major shared-memory descriptors), with an optional
+//                       reduction split whose fp32 partials are summed in a fixed order.
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..5 = epilogue
+// (each owns the 32 TMEM lanes of its warp-id quadrant).
 #include "pf_tc.h"
+
+#include <cuda.h>
+
+#include "pf_tc_prims.cuh"
 
 namespace pf {
 namespace tc {
+namespace {
 
-size_t linear_extra_workspace(int64_t, int64_t, int64_t, int64_t, bool) { return 0; }
+constexpr int kBM = 128;       // rows of the output tile = TMEM lanes
+constexpr int kBK = 64;        // contraction elements per pipeline stage (128 bytes of bf16)
+constexpr int kStages = 4;
+constexpr int kGemmThreads = 192;
+
+struct GemmCtl {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t tmem_full;
+    uint32_t tmem_base;
+    uint32_t abort;
+};
+
+struct GemmParams {
+    int M, N, K;
+    int a_mn, b_mn;          // 1 = operand stored with the M/N index contiguous
+    int kb_per_split;        // k-blocks handled by one z-slice
+    int splits;
+    void* C;                 // bf16 [M, ldc] when splits == 1
+    long long ldc;
+    float* partial;          // fp32 [splits, M, N] when splits > 1
+    unsigned int* status;
+};
+
+__device__ __forceinline__ void store_row_chunk_bf16(__nv_bfloat16* dst, const uint32_t (&v)[32], int ncols,
+                                                      bool vec_ok) {
+    if (ncols == 32 && vec_ok) {
+        uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint4 o;
+            o.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1]));
+            o.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3]));
+            o.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5]));
+            o.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]));
+            d4[q] = o;
+        }
+    } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+            if (c < ncols) dst[c] = __float2bfloat16_rn(__uint_as_float(v[c]));
+    }
+}
+__device__ __forceinline__ void store_row_chunk_f32(float* dst, const uint32_t (&v)[32], int ncols, bool vec_ok) {
+    if (ncols == 32 && vec_ok) {
+        float4* d4 = reinterpret_cast<float4*>(dst);
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            d4[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+    } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+            if (c < ncols) dst[c] = __uint_as_float(v[c]);
+    }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const GemmParams p) {
+    constexpr uint32_t kABytes = kBM * kBK * 2;          // 16 KB
+    constexpr uint32_t kBBytes = BN * kBK * 2;
+    constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+    GemmCtl* ctl = reinterpret_cast<GemmCtl*>(smem);
+    uint8_t* tiles = smem + 1024;
+    volatile uint32_t* abort_flag = &ctl->abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * BN;
+    const int nkb_total = (p.K + kBK - 1) / kBK;
+    const int kb_beg = blockIdx.z * p.kb_per_split;
+    const int kb_end = min(nkb_total, kb_beg + p.kb_per_split);
+    const int nkb = kb_end - kb_beg;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&ctl->tmem_full), 1);
+        ctl->abort = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&ctl->tmem_base), BN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % kStages;
+                const uint32_t ph = (i / kStages) & 1;
+                if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag, p.status)) break;
+                const uint32_t full = smem_u32(&ctl->full[s]);
+                const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
+                const uint32_t b_dst = a_dst + kABytes;
+                mbar_expect_tx(full, kStageBytes);
+                const int k0 = (kb_beg + i) * kBK;
+                if (p.a_mn) {
+                    tma_load_2d(a_dst, &tmA, full, m0, k0);
+                    tma_load_2d(a_dst + 8192, &tmA, full, m0 + 64, k0);
+                } else {
+                    tma_load_2d(a_dst, &tmA, full, k0, m0);
+                }
+                if (p.b_mn) {
+#pragma unroll
+                    for (int h = 0; h < BN / 64; ++h) tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, k0);
+                } else {
+                    tma_load_2d(b_dst, &tmB, full, k0, n0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(kBM, BN, p.a_mn, p.b_mn);
+            bool ok = true;
+            for (int i = 0; i < nkb && ok; ++i) {
+                const int s = i % kStages;
+                const uint32_t ph = (i / kStages) & 1;
+                ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
+                const uint32_t b_addr = a_addr + kABytes;
+                // K-major: 8-row groups 1024 B apart, 16 contraction elements = 32 B along the row.
+                // MN-major: 64-element M/N panels 8192 B apart (LBO), 8 contraction rows per
+                // 1024 B group (SBO), 16 contraction rows = 2048 B.
+                const uint64_t a_desc = p.a_mn ? make_smem_desc(a_addr, 8192, 1024) : make_smem_desc(a_addr, 16, 1024);
+                const uint64_t b_desc = p.b_mn ? make_smem_desc(b_addr, 8192, 1024) : make_smem_desc(b_addr, 16, 1024);
+                const uint32_t a_step = p.a_mn ? 2048u : 32u;
+                const uint32_t b_step = p.b_mn ? 2048u : 32u;
+#pragma unroll
+                for (int kk = 0; kk < kBK / 16; ++kk)
+                    tc_mma_bf16(tmem_base, desc_advance(a_desc, kk * a_step), desc_advance(b_desc, kk * b_step),
+                                idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&ctl->empty[s]));   // frees the stage once these MMAs have read it
+            }
+            if (ok) tc_commit(smem_u32(&ctl->tmem_full));
+        }
+    } else {
+        const int q = warp & 3;                          // TMEM lane quadrant this warp may access
+        const bool ok = mbar_wait(smem_u32(&ctl->tmem_full), 0, abort_flag, p.status);
+        tc_fence_after();
+        if (ok) {
+            const int row = m0 + q * 32 + lane;
+            const bool row_ok = row < p.M;
+            __nv_bfloat16* crow = nullptr;
+            float* prow = nullptr;
+            bool vec_ok;
+            if (p.splits > 1) {
+                prow = p.partial + (static_cast<size_t>(blockIdx.z) * p.M + (row_ok ? row : 0)) * p.N;
+                vec_ok = (p.N % 4) == 0;
+            } else {
+                crow = reinterpret_cast<__nv_bfloat16*>(p.C) + static_cast<size_t>(row_ok ? row : 0) * p.ldc;
+                vec_ok = (p.ldc % 8) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 15) == 0;
+            }
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c * 32, v);
+                tmem_ld_wait();
+                const int col = n0 + c * 32;
+                const int ncols = min(32, p.N - col);
+                if (row_ok && ncols > 0) {
+                    if (p.splits > 1) store_row_chunk_f32(prow + col, v, ncols, vec_ok);
+                    else store_row_chunk_bf16(crow + col, v, ncols, vec_ok);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, BN);
+}
+
+// ------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return static_cast<EncodeTiledFn>(nullptr);
+        return reinterpret_cast<EncodeTiledFn>(ptr);
+    }();
+    return fn;
+}
+
+// 2-D bf16 tensor map over a row-major [rows, cols] matrix with row pitch ld (elements); boxes are
+// 64 columns (128 bytes, the swizzle span) by box_rows rows; out-of-range elements read as zero.
+bool make_map_2d(CUtensorMap* map, const void* p, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+    const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tma_ok(const void* p, int64_t ld) {
+    return (reinterpret_cast<uintptr_t>(p) & 15) == 0 && (ld % 8) == 0 && ld * 2 < (1LL << 40);
+}
+
+// One operand of C = A * B.  `mn_major == false`: stored [MN, K] row-major (contraction index
+// contiguous).  `mn_major == true`: stored [K, MN] row-major (M or N index contiguous).
+struct Operand {
+    const void* p;
+    int64_t ld;
+    bool mn_major;
+};
+
+template <int BN>
+cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, dim3 grid,
+                        cudaStream_t stream) {
+    constexpr size_t smem = 1024 + 1024 + static_cast<size_t>(kStages) * (kBM * kBK * 2 + BN * kBK * 2);
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    tc_gemm_kernel<BN><<<grid, kGemmThreads, smem, stream>>>(ta, tb, p);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
+int pick_splits(int64_t M, int64_t N, int bn, int64_t K) {
+    const int64_t tiles = ceil_div(M, kBM) * ceil_div(N, bn);
+    const int64_t nkb = ceil_div(K, kBK);
+    int64_t s = kNumSMs / tiles;
+    if (s > nkb / 4) s = nkb / 4;     // at least 4 k-blocks per slice
+    if (s > 64) s = 64;
+    if (s < 1) s = 1;
+    return static_cast<int>(s);
+}
+int pick_bn(int64_t N) { return N <= 64 ? 64 : 128; }
+
+// C[M,N] (bf16, ldc) = A * B.  `partial` must hold splits*M*N floats when splits > 1.
+int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
+         int splits, float* partial, cudaStream_t stream) {
+    if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
+    const int bn = pick_bn(N);
+    CUtensorMap ta, tb;
+    const bool oka = A.mn_major ? make_map_2d(&ta, A.p, K, M, A.ld, 64) : make_map_2d(&ta, A.p, M, K, A.ld, kBM);
+    const bool okb = B.mn_major ? make_map_2d(&tb, B.p, K, N, B.ld, 64) : make_map_2d(&tb, B.p, N, K, B.ld, bn);
+    if (!oka || !okb) return PF_ERR_CUDA;
+    GemmParams p;
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.a_mn = A.mn_major; p.b_mn = B.mn_major;
+    const int64_t nkb = ceil_div(K, kBK);
+    p.kb_per_split = static_cast<int>(ceil_div(nkb, splits));
+    p.splits = static_cast<int>(ceil_div(nkb, p.kb_per_split));   // every slice gets >= 1 k-block
+    p.C = C; p.ldc = ldc; p.partial = partial;
+    p.status = device_status_ptr();
+    dim3 grid(static_cast<unsigned>(ceil_div(M, kBM)), static_cast<unsigned>(ceil_div(N, bn)),
+              static_cast<unsigned>(p.splits));
+    if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
+    cudaError_t e = bn == 64 ? launch_gemm<64>(ta, tb, p, grid, stream) : launch_gemm<128>(ta, tb, p, grid, stream);
+    if (e != cudaSuccess) return PF_ERR_CUDA;
+    if (p.splits > 1) {
+        e = splitk_reduce(partial, C, ldc, M, N, p.splits, PF_BF16, stream);
+        if (e != cudaSuccess) return PF_ERR_CUDA;
+    }
+    return PF_OK;
+}
+
+// A row-major bf16 matrix that TMA must read: used as is when 16-byte aligned with a pitch that is
+// a multiple of 8 elements, otherwise copied to `scratch` with the pitch rounded up.
+struct Staged {
+    const void* p;
+    int64_t ld;
+};
+int64_t pad8(int64_t v) { return (v + 7) / 8 * 8; }
+
+// returns 0 = usable, 1 = needs repack but no room reserved (decline), <0 never
+int stage_operand(const void* p, int64_t ld, int64_t rows, int64_t cols, char*& scratch, Staged* out,
+                  cudaStream_t stream, int* status) {
+    if (tma_ok(p, ld)) { out->p = p; out->ld = ld; return 0; }
+    if (cols % 8 == 0) return 1;   // the workspace query reserves repack room only for ragged widths
+    const int64_t ldp = pad8(cols);
+    if (repack_rows_bf16(p, ld, scratch, ldp, rows, cols, ldp, stream) != cudaSuccess) { *status = PF_ERR_CUDA; return 0; }
+    out->p = scratch; out->ld = ldp;
+    scratch += align_up(static_cast<size_t>(rows) * ldp * 2, 256);
+    return 0;
+}
+size_t repack_room(int64_t rows, int64_t cols) {
+    return cols % 8 == 0 ? 0 : align_up(static_cast<size_t>(rows) * pad8(cols) * 2, 256);
+}
+
+}  // namespace
+
+// Extra workspace of the tensor-core linear path: repack buffers for operands whose width is not a
+// multiple of 8 elements (TMA needs 16-byte row pitches), the two m x r intermediates at a padded
+// pitch, and split partials of dU / dV.
+size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool bwd) {
+    size_t b = 0;
+    b += repack_room(m, k) + repack_room(k, r) + repack_room(n, r);        // x, U, V
+    b += align_up(static_cast<size_t>(m) * pad8(r) * 2, 256);               // T at padded pitch
+    if (bwd) {
+        b += repack_room(m, n);                                             // dY
+        b += align_up(static_cast<size_t>(m) * pad8(r) * 2, 256);           // G at padded pitch
+        const int su = pick_splits(k, r, pick_bn(r), m), sv = pick_splits(n, r, pick_bn(r), m);
+        const size_t pu = su > 1 ? static_cast<size_t>(su) * k * r * 4 : 0;
+        const size_t pv = sv > 1 ? static_cast<size_t>(sv) * n * r * 4 : 0;
+        b += align_up(pu, 256) + align_up(pv, 256);
+    }
+    return b;
+}
+
 size_t conv_extra_workspace(int, int, int, int, int, int, int, int, int, int, bool) { return 0; }
-int linear_fwd(const LinearArgs&, int* handled) { *handled = 0; return PF_OK; }
-int linear_bwd(const LinearArgs&, int* handled) { *handled = 0; return PF_OK; }
+
+int linear_fwd(const LinearArgs& a, int* handled) {
+    *handled = 0;
+    if (encode_fn() == nullptr) return PF_OK;
+    int st = PF_OK;
+    char* scratch = a.ws;
+    Staged x, U, V;
+    if (stage_operand(a.x, a.ldx, a.m, a.k, scratch, &x, a.stream, &st)) return PF_OK;
+    if (stage_operand(a.U, a.ldu, a.k, a.r, scratch, &U, a.stream, &st)) return PF_OK;
+    if (stage_operand(a.V, a.ldv, a.n, a.r, scratch, &V, a.stream, &st)) return PF_OK;
+    if (st != PF_OK) return st;
+    *handled = 1;
+    // T: written straight into the stash when TMA can read it back, else into padded scratch
+    void* T = scratch;
+    int64_t ldT = pad8(a.r);
+    const bool stash_direct = a.T && tma_ok(a.T, a.ldt);
+    if (stash_direct) { T = a.T; ldT = a.ldt; }
+    st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, T, ldT, 1, nullptr, a.stream);
+    if (st != PF_OK) return st;
+    if (a.T && !stash_direct &&
+        repack_rows_bf16(T, ldT, a.T, a.ldt, a.m, a.r, a.r, a.stream) != cudaSuccess)
+        return PF_ERR_CUDA;
+    return gemm({T, ldT, false}, {V.p, V.ld, false}, a.m, a.n, a.r, a.y, a.ldy, 1, nullptr, a.stream);
+}
+
+int linear_bwd(const LinearArgs& a, int* handled) {
+    *handled = 0;
+    if (encode_fn() == nullptr) return PF_OK;
+    int st = PF_OK;
+    char* scratch = a.ws;
+    Staged x, U, V, dY, T;
+    if (stage_operand(a.x, a.ldx, a.m, a.k, scratch, &x, a.stream, &st)) return PF_OK;
+    if (stage_operand(a.U, a.ldu, a.k, a.r, scratch, &U, a.stream, &st)) return PF_OK;
+    if (stage_operand(a.V, a.ldv, a.n, a.r, scratch, &V, a.stream, &st)) return PF_OK;
+    if (stage_operand(a.dY, a.lddy, a.m, a.n, scratch, &dY, a.stream, &st)) return PF_OK;
+    if (st != PF_OK) return st;
+    char* Tbuf = scratch;
+    scratch += align_up(static_cast<size_t>(a.m) * pad8(a.r) * 2, 256);
+    if (a.T) {
+        if (tma_ok(a.T, a.ldt)) { T.p = a.T; T.ld = a.ldt; }
+        else if (a.r % 8 == 0) return PF_OK;   // odd pitch on an even width: FMA path
+        else {
+            if (repack_rows_bf16(a.T, a.ldt, Tbuf, pad8(a.r), a.m, a.r, pad8(a.r), a.stream) != cudaSuccess)
+                return PF_ERR_CUDA;
+            T.p = Tbuf; T.ld = pad8(a.r);
+        }
+    }
+    *handled = 1;
+    if (!a.T) {
+        st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, Tbuf, pad8(a.r), 1, nullptr, a.stream);
+        if (st != PF_OK) return st;
+        T.p = Tbuf; T.ld = pad8(a.r);
+    }
+    char* G = scratch;
+    const int64_t ldG = pad8(a.r);
+    scratch += align_up(static_cast<size_t>(a.m) * ldG * 2, 256);
+    const int su = pick_splits(a.k, a.r, pick_bn(a.r), a.m), sv = pick_splits(a.n, a.r, pick_bn(a.r), a.m);
+    float* pu = reinterpret_cast<float*>(scratch);
+    scratch += align_up(su > 1 ? static_cast<size_t>(su) * a.k * a.r * 4 : 0, 256);
+    float* pv = reinterpret_cast<float*>(scratch);
+    // G = dY V ; dX = G U^T ; dU = x^T G ; dV = dY^T T
+    st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG, 1, nullptr, a.stream);
+    if (st != PF_OK) return st;
+    if (a.dX) {
+        st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
+        if (st != PF_OK) return st;
+    }
+    st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream);
+    if (st != PF_OK) return st;
+    return gemm({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, a.stream);
+}
+
 int conv_fwd(const ConvArgs&, int* handled) { *handled = 0; return PF_OK; }
 int conv_bwd(const ConvArgs&, int* handled) { *handled = 0; return PF_OK; }
 
