@@ -86,6 +86,31 @@ int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The same forward for callers that cannot allocate device memory and therefore have no
+ * workspace to pass: latency-critical host paths where cudaMalloc is forbidden because it
+ * synchronises the device, plug-ins that are handed tensors but no allocator, and processes
+ * whose device memory is already fully committed to a pool they do not control.
+ * (The paper has no counterpart; this is a deployment variant.)
+ *
+ * Identical to pf_lowrank_linear_fwd except that the scratch is a fixed array inside the
+ * library image (PF_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the
+ * process exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Problems whose pf_lowrank_linear_workspace(m, k, n, r, dtype, 0) exceeds
+ *     PF_STATIC_SCRATCH_BYTES are rejected with PF_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address (a one-time
+ *     set-up with that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the previous call
+ *     left in it: two calls that may overlap on the GPU (different streams) race and must be
+ *     ordered by the caller.  Nothing in the array has to be cleared between calls.
+ * pf_static_scratch_bytes() returns PF_STATIC_SCRATCH_BYTES as compiled. */
+#define PF_STATIC_SCRATCH_BYTES (8u << 20)
+int pf_lowrank_linear_fwd_static(const void* x, int64_t ldx, const void* U, int64_t ldu,
+                                 const void* V, int64_t ldv, void* y, int64_t ldy,
+                                 void* T_stash, int64_t ldt,
+                                 int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                                 void* cuda_stream);
+size_t pf_static_scratch_bytes(void);
+
 /* Gradients of the layer above for an upstream gradient dY [m, n] (chain rule on
  * y = (xU)V^T; plain sums over the m rows, no averaging):
  *   G  = dY V           [m, r]  (kept on chip / in workspace)

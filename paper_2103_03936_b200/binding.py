@@ -44,6 +44,10 @@ def lib() -> ctypes.CDLL:
         L.pf_lowrank_linear_fwd.restype = ci
         L.pf_lowrank_linear_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                             i64, i64, i64, i64, ci, vp, sz, vp]
+        L.pf_lowrank_linear_fwd_static.restype = ci
+        L.pf_lowrank_linear_fwd_static.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
+                                                   i64, i64, i64, i64, ci, vp]
+        L.pf_static_scratch_bytes.restype = sz
         L.pf_lowrank_linear_bwd.restype = ci
         L.pf_lowrank_linear_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                             vp, i64, vp, i64, vp, i64,
@@ -150,6 +154,28 @@ def pf_lowrank_linear_fwd(x, U, V, *, y=None, T_stash=None, want_stash=False, wo
         return _Prepared(lib().pf_lowrank_linear_fwd, args, "pf_lowrank_linear_fwd", (x, U, V, y, T_stash, ws)), out
     _check(lib().pf_lowrank_linear_fwd(*args), "pf_lowrank_linear_fwd")
     return out
+
+
+def pf_static_scratch_bytes() -> int:
+    return int(lib().pf_static_scratch_bytes())
+
+
+def pf_lowrank_linear_fwd_static(x, U, V, *, y, T_stash=None, stream=None):
+    """y = (x U) V^T for callers that cannot allocate: the scratch is a fixed array inside the
+    library, so the caller passes inputs and outputs only (y is required; nothing is allocated
+    here either).  Raises PfError(PF_ERR_WORKSPACE) when the problem does not fit the array.
+    Calls on one device share that array: do not let two of them overlap on the GPU."""
+    dt = _dtype_code(x)
+    m, k = x.shape
+    n, r = V.shape
+    if U.shape != (k, r):
+        raise ValueError("U must be [k, r] and V [n, r]")
+    st = lib().pf_lowrank_linear_fwd_static(
+        _ptr(x), _mat(x, "x"), _ptr(U), _mat(U, "U"), _ptr(V), _mat(V, "V"), _ptr(y), _mat(y, "y"),
+        _ptr(T_stash), _mat(T_stash, "T_stash") if T_stash is not None else 0,
+        m, k, n, r, dt, _stream(stream))
+    _check(st, "pf_lowrank_linear_fwd_static")
+    return (y, T_stash) if T_stash is not None else y
 
 
 def pf_lowrank_linear_bwd(x, U, V, dY, *, T_stash=None, need_dX=True, dX=None, dU=None, dV=None,
