@@ -12,6 +12,7 @@
 
 #include <cuda.h>
 
+#include "pf_tc_host.h"
 #include "pf_tc_prims.cuh"
 
 namespace pf {
@@ -203,41 +204,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ------------------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return static_cast<EncodeTiledFn>(nullptr);
-        return reinterpret_cast<EncodeTiledFn>(ptr);
-    }();
-    return fn;
-}
-
-// 2-D bf16 tensor map over a row-major [rows, cols] matrix with row pitch ld (elements); boxes are
-// 64 columns (128 bytes, the swizzle span) by box_rows rows; out-of-range elements read as zero.
-bool make_map_2d(CUtensorMap* map, const void* p, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
-    const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
-    const cuuint32_t estr[2] = {1u, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-bool tma_ok(const void* p, int64_t ld) {
-    return (reinterpret_cast<uintptr_t>(p) & 15) == 0 && (ld % 8) == 0 && ld * 2 < (1LL << 40);
-}
-
 // One operand of C = A * B.  `mn_major == false`: stored [MN, K] row-major (contraction index
 // contiguous).  `mn_major == true`: stored [K, MN] row-major (M or N index contiguous).
 struct Operand {
@@ -324,6 +290,9 @@ int stage_operand(const void* p, int64_t ld, int64_t rows, int64_t cols, char*& 
     scratch += align_up(static_cast<size_t>(rows) * ldp * 2, 256);
     return 0;
 }
+// The fused chain pays off once there are enough 128-row tiles to fill the machine.
+bool use_chain(int64_t m) { return m >= 2048; }
+
 size_t repack_room(int64_t rows, int64_t cols) {
     return cols % 8 == 0 ? 0 : align_up(static_cast<size_t>(rows) * pad8(cols) * 2, 256);
 }
@@ -366,12 +335,21 @@ int linear_fwd(const LinearArgs& a, int* handled) {
     int64_t ldT = pad8(a.r);
     const bool stash_direct = a.T && tma_ok(a.T, a.ldt);
     if (stash_direct) { T = a.T; ldT = a.ldt; }
-    st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, T, ldT, 1, nullptr, a.stream);
+    ChainPlan plan;
+    if (use_chain(a.m) && tma_ok(a.y, a.ldy) && chain_plan(a.m, a.k, a.n, a.r, true, &plan)) {
+        // one fused kernel; the intermediate leaves the chip only if a stash was asked for
+        st = chain(x.p, x.ld, a.m, a.k, U.p, U.ld, a.r, V.p, V.ld, a.n, a.y, a.ldy, a.T ? T : nullptr, ldT,
+                   a.stream);
+    } else {
+        st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, T, ldT, 1, nullptr, a.stream);
+        if (st != PF_OK) return st;
+        st = gemm({T, ldT, false}, {V.p, V.ld, false}, a.m, a.n, a.r, a.y, a.ldy, 1, nullptr, a.stream);
+    }
     if (st != PF_OK) return st;
     if (a.T && !stash_direct &&
         repack_rows_bf16(T, ldT, a.T, a.ldt, a.m, a.r, a.r, a.stream) != cudaSuccess)
         return PF_ERR_CUDA;
-    return gemm({T, ldT, false}, {V.p, V.ld, false}, a.m, a.n, a.r, a.y, a.ldy, 1, nullptr, a.stream);
+    return PF_OK;
 }
 
 int linear_bwd(const LinearArgs& a, int* handled) {
@@ -410,11 +388,17 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     scratch += align_up(su > 1 ? static_cast<size_t>(su) * a.k * a.r * 4 : 0, 256);
     float* pv = reinterpret_cast<float*>(scratch);
     // G = dY V ; dX = G U^T ; dU = x^T G ; dV = dY^T T
-    st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG, 1, nullptr, a.stream);
-    if (st != PF_OK) return st;
-    if (a.dX) {
-        st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
+    ChainPlan plan;
+    if (use_chain(a.m) && (!a.dX || tma_ok(a.dX, a.lddx)) && chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan)) {
+        st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream);
         if (st != PF_OK) return st;
+    } else {
+        st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG, 1, nullptr, a.stream);
+        if (st != PF_OK) return st;
+        if (a.dX) {
+            st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
+            if (st != PF_OK) return st;
+        }
     }
     st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream);
     if (st != PF_OK) return st;

@@ -29,6 +29,16 @@ struct ConvArgs {
     cudaStream_t stream;
 };
 
+// Fused chain kernel (pf_tc_chain.cu): out = (A * B1) * B2^T with the intermediate on chip.
+struct ChainPlan {
+    int r_pad, num_stages, stage_bytes, nsplit, tiles_per_split, row_tiles;
+    size_t smem;
+};
+bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan);
+int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
+          const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
+          cudaStream_t stream);
+
 size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool bwd);
 size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
                             int pad, bool bwd);

@@ -1,0 +1,336 @@
+// Fused two-GEMM chain for sm_100a:   out[M, N2] = (A[M, K1] * B1[K1, r]) * B2[N2, r]^T
+// with the M x r intermediate kept on chip (fp32 in tensor memory, then bf16 in shared memory)
+// and optionally also written out once (the stash).  It serves both
+//   forward   y  = (x  U) V^T      A = x,  B1 = U [k, r],  B2 = V [n, r]
+//   backward  dX = (dY V) U^T      A = dY, B1 = V [n, r],  B2 = U [k, r]
+// of the factorized linear layer.
+//
+// One CTA owns one 128-row tile of A (and a contiguous range of 128-column output tiles when the
+// grid splits N2 to fill the machine; each split then recomputes the intermediate).
+//   phase 1  T = A * B1: TMA ring over K1 in 64-element blocks; A tile is a K-major operand,
+//            the B1 tile [64 x r] is an MN-major operand (r contiguous in memory); fp32
+//            accumulator of r columns in TMEM.
+//   switch   the four epilogue warps read T from TMEM, round to bf16 and lay it out in shared
+//            memory as the K-major (128-byte swizzled) A operand of phase 2; the same bytes are
+//            what TMA stores as the stash.
+//   phase 2  for each 128-column tile: out_tile = T * B2_tile^T with B2 tiles streamed through
+//            the same ring; accumulators double-buffered in TMEM so the MMAs of tile j+1 overlap
+//            the epilogue of tile j; the epilogue stages bf16 rows in swizzled shared memory and
+//            writes them with TMA stores (coalesced, clipped at the matrix edge).
+// Shared memory: control block | T (r_pad x 256 B) | ring of stages (16 KB A or B2 tile + r_pad x
+// 128 B B1 tile).  In phase 2 the B1 part of every stage is idle and serves as store staging.
+#include <cuda.h>
+
+#include "pf_tc.h"
+#include "pf_tc_host.h"
+#include "pf_tc_prims.cuh"
+
+namespace pf {
+namespace tc {
+namespace {
+
+constexpr int kMaxStages = 8;
+constexpr int kChainThreads = 192;
+constexpr uint32_t kTileBytes = 16384;      // 128 rows x 64 bf16
+
+struct ChainCtl {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t t_full;        // phase-1 accumulator complete
+    uint64_t t_ready;       // bf16 T is in shared memory (one arrival per epilogue warp)
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort;
+};
+
+struct ChainParams {
+    int M, K1, N2;
+    int r_pad;              // r rounded up to a multiple of 64, <= 384
+    int num_stages;
+    int stage_bytes;        // 16384 + r_pad * 128
+    int tiles_per_split;    // 128-column output tiles per blockIdx.y (0: phase 1 only)
+    int store_T;
+    unsigned int* status;
+};
+
+__device__ __forceinline__ uint4 pack8(const uint32_t* v) {
+    uint4 o;
+    o.x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+    o.y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+    o.z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+    o.w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+    return o;
+}
+
+__global__ void __launch_bounds__(kChainThreads, 1)
+tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB1,
+                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmOut,
+                const __grid_constant__ CUtensorMap tmT, const ChainParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+    ChainCtl* ctl = reinterpret_cast<ChainCtl*>(smem);
+    const uint32_t t_smem = smem_u32(smem + 1024);
+    const uint32_t ring = t_smem + static_cast<uint32_t>(p.r_pad) * 256u;
+    volatile uint32_t* abort_flag = &ctl->abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * 128;
+    const int nt_total = (p.N2 + 127) / 128;
+    const int t_beg = blockIdx.y * p.tiles_per_split;
+    const int ntile = max(0, min(nt_total, t_beg + p.tiles_per_split) - t_beg);
+    const int nkb1 = (p.K1 + 63) / 64;
+    const int nkb2 = p.r_pad / 64;
+    const int NS = p.num_stages;
+    const uint32_t S = static_cast<uint32_t>(p.stage_bytes);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&ctl->t_full), 1);
+        mbar_init(smem_u32(&ctl->t_ready), 4);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
+        }
+        ctl->abort = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB1);
+        tma_prefetch_desc(&tmB2);
+        tma_prefetch_desc(&tmOut);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&ctl->tmem_base), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int kb = 0; kb < nkb1 && ok; ++kb, ++it) {
+                const int s = it % NS;
+                ok = mbar_wait(smem_u32(&ctl->empty[s]), ((it / NS) & 1) ^ 1u, abort_flag, p.status);
+                if (!ok) break;
+                const uint32_t full = smem_u32(&ctl->full[s]);
+                const uint32_t dst = ring + s * S;
+                mbar_expect_tx(full, kTileBytes + static_cast<uint32_t>(p.r_pad) * 128u);
+                tma_load_2d(dst, &tmA, full, kb * 64, m0);
+                for (int q = 0; q < nkb2; ++q)
+                    tma_load_2d(dst + kTileBytes + q * 8192, &tmB1, full, q * 64, kb * 64);
+            }
+            for (int j = 0; j < ntile && ok; ++j) {
+                const int n0 = (t_beg + j) * 128;
+                for (int kb = 0; kb < nkb2; ++kb, ++it) {
+                    const int s = it % NS;
+                    ok = mbar_wait(smem_u32(&ctl->empty[s]), ((it / NS) & 1) ^ 1u, abort_flag, p.status);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctl->full[s]);
+                    mbar_expect_tx(full, kTileBytes);
+                    tma_load_2d(ring + s * S, &tmB2, full, kb * 64, n0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            const int n1a = min(256, p.r_pad), n1b = p.r_pad - n1a;
+            const uint32_t idesc_a = make_idesc_bf16(128, n1a, 0, 1);
+            const uint32_t idesc_b = make_idesc_bf16(128, n1b > 0 ? n1b : 64, 0, 1);
+            for (int kb = 0; kb < nkb1 && ok; ++kb, ++it) {
+                const int s = it % NS;
+                ok = mbar_wait(smem_u32(&ctl->full[s]), (it / NS) & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = ring + s * S;
+                const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
+                const uint64_t b_desc = make_smem_desc(a_addr + kTileBytes, 8192, 1024);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint32_t acc = (kb > 0 || kk > 0) ? 1u : 0u;
+                    tc_mma_bf16(tmem, desc_advance(a_desc, kk * 32), desc_advance(b_desc, kk * 2048), idesc_a, acc);
+                    if (n1b > 0)
+                        tc_mma_bf16(tmem + 256, desc_advance(a_desc, kk * 32),
+                                    desc_advance(b_desc, 4 * 8192 + kk * 2048), idesc_b, acc);
+                }
+                tc_commit(smem_u32(&ctl->empty[s]));
+            }
+            if (ok) tc_commit(smem_u32(&ctl->t_full));
+            if (ok) ok = mbar_wait(smem_u32(&ctl->t_ready), 0, abort_flag, p.status);
+            tc_fence_after();
+            const bool stash = ok && p.store_T && blockIdx.y == 0;
+            if (stash) {
+                for (int q = 0; q < nkb2; ++q) tma_store_2d(&tmT, t_smem + q * kTileBytes, q * 64, m0);
+                tma_store_commit();
+            }
+            const uint32_t idesc2 = make_idesc_bf16(128, 128, 0, 0);
+            for (int j = 0; j < ntile && ok; ++j) {
+                const int b = j & 1;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), ((j >> 1) & 1) ^ 1u, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                for (int kb = 0; kb < nkb2; ++kb, ++it) {
+                    const int s = it % NS;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), (it / NS) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t a_desc = make_smem_desc(t_smem + kb * kTileBytes, 16, 1024);
+                    const uint64_t b_desc = make_smem_desc(ring + s * S, 16, 1024);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma_bf16(tmem + b * 128, desc_advance(a_desc, kk * 32), desc_advance(b_desc, kk * 32),
+                                    idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&ctl->empty[s]));
+                }
+                if (ok) tc_commit(smem_u32(&ctl->acc_full[b]));
+            }
+            if (stash) tma_store_wait_read<0>();
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>(q * 32) << 16);
+        bool ok = mbar_wait(smem_u32(&ctl->t_full), 0, abort_flag, p.status);
+        tc_fence_after();
+        if (ok) {
+            const uint32_t sw = static_cast<uint32_t>(row & 7);
+            for (int c = 0; c < p.r_pad / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(lane_base + c * 32, v);
+                tmem_ld_wait();
+                const uint32_t panel = t_smem + (c >> 1) * kTileBytes + row * 128;
+                const uint32_t cb = (c & 1) * 4;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) st_shared_v4(panel + (((cb + t) ^ sw) << 4), pack8(v + 8 * t));
+            }
+            tc_fence_before();
+            fence_proxy_async_smem();
+        }
+        __syncwarp();
+        if (ok && lane == 0) mbar_arrive(smem_u32(&ctl->t_ready));
+
+        const int pieces = p.r_pad / 64;   // 8 KB staging pieces in the idle B1 part of each stage
+        bool stored = false;
+        for (int j = 0; j < ntile && ok; ++j) {
+            const int b = j & 1;
+            ok = mbar_wait(smem_u32(&ctl->acc_full[b]), (j >> 1) & 1, abort_flag, p.status);
+            tc_fence_after();
+            if (!ok) break;
+            const int wb = q * 2 + b;
+            const uint32_t stg = ring + (wb / pieces) * S + kTileBytes + (wb % pieces) * 8192;
+            if (lane == 0) tma_store_wait_read<1>();   // the store that used this buffer two tiles ago
+            __syncwarp();
+            const uint32_t sw = static_cast<uint32_t>(lane & 7);
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(lane_base + b * 128 + c * 32, v);
+                tmem_ld_wait();
+                const uint32_t prow = stg + (c >> 1) * 4096 + lane * 128;
+                const uint32_t cb = (c & 1) * 4;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) st_shared_v4(prow + (((cb + t) ^ sw) << 4), pack8(v + 8 * t));
+            }
+            tc_fence_before();
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                const int n0 = (t_beg + j) * 128, r0 = m0 + q * 32;
+                if (r0 < p.M) {
+                    tma_store_2d(&tmOut, stg, n0, r0);
+                    if (n0 + 64 < p.N2) tma_store_2d(&tmOut, stg + 4096, n0 + 64, r0);
+                }
+                tma_store_commit();
+                stored = true;
+            }
+        }
+        if (lane == 0 && stored) tma_store_wait_read<0>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+}  // namespace
+
+// Shape envelope of the fused kernel and its launch geometry.
+bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan) {
+    const int64_t r_pad = (r + 63) / 64 * 64;
+    if (r_pad > 384 || M > 0x7fffffff || K1 > 0x7fffffff || N2 > 0x7fffffff) return false;
+    const int64_t stage = kTileBytes + r_pad * 128;
+    const int64_t budget = 227 * 1024 - 2048 - r_pad * 256;
+    int64_t ns = budget / stage;
+    if (ns > kMaxStages) ns = kMaxStages;
+    if (ns < 2 || ns * (r_pad / 64) < 8) return false;
+    const int64_t row_tiles = ceil_div(M, 128), nt = ceil_div(N2, 128);
+    // Split N2 over blockIdx.y while that shortens the critical path of a CTA (each split repeats
+    // phase 1, cost ~ K1; phase 2 costs ~ N2 / split) and the grid still fits one wave.
+    int64_t best = 1;
+    if (has_out) {
+        double best_cost = 1e30;
+        for (int64_t s = 1; s <= nt && (s == 1 || row_tiles * s <= kNumSMs); ++s) {
+            const double waves = static_cast<double>(ceil_div(row_tiles * s, kNumSMs));
+            const double cost = waves * (static_cast<double>(K1) + 128.0 * ceil_div(nt, s));
+            if (cost < best_cost * 0.97) { best_cost = cost; best = s; }
+        }
+    }
+    plan->r_pad = static_cast<int>(r_pad);
+    plan->num_stages = static_cast<int>(ns);
+    plan->stage_bytes = static_cast<int>(stage);
+    plan->nsplit = static_cast<int>(has_out ? best : 1);
+    plan->tiles_per_split = has_out ? static_cast<int>(ceil_div(nt, best)) : 0;
+    plan->nsplit = has_out ? static_cast<int>(ceil_div(nt, plan->tiles_per_split)) : 1;
+    plan->smem = static_cast<size_t>(2048 + r_pad * 256 + ns * stage);
+    plan->row_tiles = static_cast<int>(row_tiles);
+    return true;
+}
+
+// out may be null (phase 1 only: T is written and nothing else).  All pointers must satisfy tma_ok.
+int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
+          const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
+          cudaStream_t stream) {
+    ChainPlan plan;
+    if (!chain_plan(M, K1, N2, r, out != nullptr, &plan)) return PF_ERR_UNSUPPORTED;
+    CUtensorMap ta, tb1, tb2, to, tt;
+    bool ok = make_map_2d(&ta, A, M, K1, lda, 128) && make_map_2d(&tb1, B1, K1, r, ldb1, 64) &&
+              make_map_2d(&tb2, B2, N2, r, ldb2, 128);
+    ok = ok && (out ? make_map_2d(&to, out, M, N2, ldo, 32) : make_map_2d(&to, A, M, K1, lda, 32));
+    ok = ok && (T ? make_map_2d(&tt, T, M, r, ldt, 128) : make_map_2d(&tt, A, M, K1, lda, 128));
+    if (!ok) return PF_ERR_CUDA;
+    ChainParams p;
+    p.M = static_cast<int>(M); p.K1 = static_cast<int>(K1); p.N2 = static_cast<int>(N2);
+    p.r_pad = plan.r_pad; p.num_stages = plan.num_stages; p.stage_bytes = plan.stage_bytes;
+    p.tiles_per_split = plan.tiles_per_split; p.store_T = T != nullptr;
+    p.status = device_status_ptr();
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        if (cudaFuncSetAttribute(tc_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess)
+            return PF_ERR_CUDA;
+        configured[dev] = true;
+    }
+    dim3 grid(static_cast<unsigned>(plan.row_tiles), static_cast<unsigned>(plan.nsplit), 1);
+    tc_chain_kernel<<<grid, kChainThreads, plan.smem, stream>>>(ta, tb1, tb2, to, tt, p);
+    if (cudaGetLastError() != cudaSuccess) return PF_ERR_CUDA;
+    count_launch();
+    return PF_OK;
+}
+
+}  // namespace tc
+}  // namespace pf

@@ -71,6 +71,16 @@ def test_multi_tile_ragged(dtype, m, k, n, r):
     run_case(wl.LinearCase("rag", m, k, n, r, dtype, 7))
 
 
+@pytest.mark.parametrize("m,k,n,r", [(2100, 200, 328, 40), (2048, 1504, 520, 376), (2500, 136, 72, 200),
+                                     (4100, 72, 1000, 130), (2048, 64, 64, 256), (2304, 520, 264, 320),
+                                     (2050, 100, 130, 33)])
+def test_fused_chain_envelope(m, k, n, r):
+    """m >= 2048 takes the fused two-GEMM kernel: every rank padding (64..384), ragged row tile,
+    ragged k / n tails, with and without stash and dX."""
+    run_case(wl.LinearCase("chain", m, k, n, r, wl.BF16, 13))
+    run_case(wl.LinearCase("chain", m, k, n, r, wl.BF16, 14), stash=False, need_dX=False)
+
+
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_leading_dimensions_and_padding_untouched(dtype):
     run_case(wl.LinearCase("ld", 200, 72, 136, 24, dtype, 8), ld_pad=8)
