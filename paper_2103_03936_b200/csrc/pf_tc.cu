@@ -115,11 +115,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
+    // Producer and MMA issuer are each one thread chosen with elect.sync that runs its whole role
+    // (a thread singled out by a lane-id test issues TMA / tcgen05 instructions several times slower).
     if (warp == 0) {
-        if (lane == 0) {
+        if (elect_one()) {
+            uint32_t s = 0, ph = 0;
             for (int i = 0; i < nkb; ++i) {
-                const int s = i % kStages;
-                const uint32_t ph = (i / kStages) & 1;
                 if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag, p.status)) break;
                 const uint32_t full = smem_u32(&ctl->full[s]);
                 const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
@@ -138,38 +139,38 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 } else {
                     tma_load_2d(b_dst, &tmB, full, k0, n0);
                 }
+                if (++s == kStages) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (elect_one()) {
             const uint32_t idesc = make_idesc_bf16(kBM, BN, p.a_mn, p.b_mn);
+            // K-major: 8-row groups 1024 B apart, 16 contraction elements = 32 B along the row.
+            // MN-major: 64-element M/N panels 8192 B apart (LBO), 8 contraction rows per
+            // 1024 B group (SBO), 16 contraction rows = 2048 B.
+            const uint32_t a_step = p.a_mn ? 128u : 2u, b_step = p.b_mn ? 128u : 2u;   // in 16-byte units
+            uint32_t s = 0, ph = 0;
             bool ok = true;
-            for (int i = 0; i < nkb && ok; ++i) {
-                const int s = i % kStages;
-                const uint32_t ph = (i / kStages) & 1;
+            for (int i = 0; i < nkb; ++i) {
                 ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
                 const uint32_t b_addr = a_addr + kABytes;
-                // K-major: 8-row groups 1024 B apart, 16 contraction elements = 32 B along the row.
-                // MN-major: 64-element M/N panels 8192 B apart (LBO), 8 contraction rows per
-                // 1024 B group (SBO), 16 contraction rows = 2048 B.
                 const uint64_t a_desc = p.a_mn ? make_smem_desc(a_addr, 8192, 1024) : make_smem_desc(a_addr, 16, 1024);
                 const uint64_t b_desc = p.b_mn ? make_smem_desc(b_addr, 8192, 1024) : make_smem_desc(b_addr, 16, 1024);
-                const uint32_t a_step = p.a_mn ? 2048u : 32u;
-                const uint32_t b_step = p.b_mn ? 2048u : 32u;
-#pragma unroll
-                for (int kk = 0; kk < kBK / 16; ++kk)
-                    tc_mma_bf16(tmem_base, desc_advance(a_desc, kk * a_step), desc_advance(b_desc, kk * b_step),
-                                idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                tc_mma_bf16(tmem_base, a_desc, b_desc, idesc, i > 0 ? 1u : 0u);
+                tc_mma_bf16(tmem_base, a_desc + a_step, b_desc + b_step, idesc, 1u);
+                tc_mma_bf16(tmem_base, a_desc + 2 * a_step, b_desc + 2 * b_step, idesc, 1u);
+                tc_mma_bf16(tmem_base, a_desc + 3 * a_step, b_desc + 3 * b_step, idesc, 1u);
                 tc_commit(smem_u32(&ctl->empty[s]));   // frees the stage once these MMAs have read it
+                if (++s == kStages) { s = 0; ph ^= 1u; }
             }
             if (ok) tc_commit(smem_u32(&ctl->tmem_full));
         }
     } else {
         const int q = warp & 3;                          // TMEM lane quadrant this warp may access
-        const bool ok = mbar_wait(smem_u32(&ctl->tmem_full), 0, abort_flag, p.status);
+        const bool ok = mbar_wait_warp(smem_u32(&ctl->tmem_full), 0, abort_flag, p.status);
         tc_fence_after();
         if (ok) {
             const int row = m0 + q * 32 + lane;

@@ -31,7 +31,7 @@ struct ConvArgs {
 
 // Fused chain kernel (pf_tc_chain.cu): out = (A * B1) * B2^T with the intermediate on chip.
 struct ChainPlan {
-    int r_pad, num_stages, stage_bytes, nsplit, tiles_per_split, row_tiles;
+    int r_pad, num_stages, stage_bytes, nsplit, tiles_per_split, row_tiles, boxes_per_stage, staging_off;
     size_t smem;
 };
 bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan);

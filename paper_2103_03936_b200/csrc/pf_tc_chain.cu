@@ -32,14 +32,15 @@ namespace {
 constexpr int kMaxStages = 8;
 constexpr int kChainThreads = 192;
 constexpr uint32_t kTileBytes = 16384;      // 128 rows x 64 bf16
+constexpr int kAccBufs = 4;                 // 4 x 128 TMEM columns of phase-2 accumulators
 
 struct ChainCtl {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
     uint64_t t_full;        // phase-1 accumulator complete
     uint64_t t_ready;       // bf16 T is in shared memory (one arrival per epilogue warp)
-    uint64_t acc_full[2];
-    uint64_t acc_empty[2];
+    uint64_t acc_full[kAccBufs];
+    uint64_t acc_empty[kAccBufs];
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -51,6 +52,8 @@ struct ChainParams {
     int stage_bytes;        // 16384 + r_pad * 128
     int tiles_per_split;    // 128-column output tiles per blockIdx.y (0: phase 1 only)
     int store_T;
+    int boxes_per_stage;    // phase 2: B2 boxes (16 KB each) loaded per ring stage
+    int staging_off;        // byte offset (from the 1 KB-aligned base) of dedicated store staging, 0 = none
     unsigned int* status;
 };
 
@@ -62,6 +65,14 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* v) {
     o.w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
     return o;
 }
+
+// Ring position: stage index, its byte offset and the phase bit, advanced without divisions.
+struct RingPos {
+    uint32_t s = 0, off = 0, ph = 0;
+    __device__ __forceinline__ void advance(uint32_t ns, uint32_t stage_bytes) {
+        if (++s == ns) { s = 0; off = 0; ph ^= 1u; } else { off += stage_bytes; }
+    }
+};
 
 __global__ void __launch_bounds__(kChainThreads, 1)
 tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB1,
@@ -82,17 +93,18 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int ntile = max(0, min(nt_total, t_beg + p.tiles_per_split) - t_beg);
     const int nkb1 = (p.K1 + 63) / 64;
     const int nkb2 = p.r_pad / 64;
-    const int NS = p.num_stages;
+    const uint32_t NS = static_cast<uint32_t>(p.num_stages);
     const uint32_t S = static_cast<uint32_t>(p.stage_bytes);
+    const int bps = p.boxes_per_stage;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) {
+        for (uint32_t s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->t_full), 1);
         mbar_init(smem_u32(&ctl->t_ready), 4);
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
         }
@@ -109,60 +121,78 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
+    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
 
+    // Producer and MMA issuer are each ONE thread chosen with elect.sync, running its whole role.
+    // (A thread singled out by a lane-id test issues tcgen05 / TMA instructions several times
+    // slower, and the issuing thread's own instruction latency is on the critical path, so the
+    // loops below carry running offsets instead of recomputing them.)
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int it = 0;
+        if (elect_one()) {
+            // -------------------------------------------------------------- TMA producer
+            RingPos rp;
             bool ok = true;
-            for (int kb = 0; kb < nkb1 && ok; ++kb, ++it) {
-                const int s = it % NS;
-                ok = mbar_wait(smem_u32(&ctl->empty[s]), ((it / NS) & 1) ^ 1u, abort_flag, p.status);
+            // Phase 2 streams B2 tiles that nobody has touched yet; have L2 fetch them while phase 1
+            // runs.  The CTAs that share these tiles each ask for a different one.
+            if (ntile > 0) {
+                const int n0 = (t_beg + static_cast<int>(blockIdx.x) % ntile) * 128;
+                for (int q = 0; q < nkb2; ++q) tma_prefetch_l2_2d(&tmB2, q * 64, n0);
+            }
+            const uint32_t tx1 = kTileBytes + static_cast<uint32_t>(p.r_pad) * 128u;
+            for (int kb = 0; kb < nkb1; ++kb) {
+                ok = mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status);
                 if (!ok) break;
-                const uint32_t full = smem_u32(&ctl->full[s]);
-                const uint32_t dst = ring + s * S;
-                mbar_expect_tx(full, kTileBytes + static_cast<uint32_t>(p.r_pad) * 128u);
+                const uint32_t full = full0 + 8 * rp.s;
+                const uint32_t dst = ring + rp.off;
+                mbar_expect_tx(full, tx1);
                 tma_load_2d(dst, &tmA, full, kb * 64, m0);
                 for (int q = 0; q < nkb2; ++q)
                     tma_load_2d(dst + kTileBytes + q * 8192, &tmB1, full, q * 64, kb * 64);
+                rp.advance(NS, S);
             }
             for (int j = 0; j < ntile && ok; ++j) {
                 const int n0 = (t_beg + j) * 128;
-                for (int kb = 0; kb < nkb2; ++kb, ++it) {
-                    const int s = it % NS;
-                    ok = mbar_wait(smem_u32(&ctl->empty[s]), ((it / NS) & 1) ^ 1u, abort_flag, p.status);
+                for (int kb = 0; kb < nkb2; kb += bps) {
+                    const int nb = min(bps, nkb2 - kb);
+                    ok = mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
-                    const uint32_t full = smem_u32(&ctl->full[s]);
-                    mbar_expect_tx(full, kTileBytes);
-                    tma_load_2d(ring + s * S, &tmB2, full, kb * 64, n0);
+                    const uint32_t full = full0 + 8 * rp.s;
+                    mbar_expect_tx(full, kTileBytes * nb);
+                    for (int q = 0; q < nb; ++q)
+                        tma_load_2d(ring + rp.off + q * kTileBytes, &tmB2, full, (kb + q) * 64, n0);
+                    rp.advance(NS, S);
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            int it = 0;
+        if (elect_one()) {
+            // -------------------------------------------------------------- MMA issuer
+            RingPos rp;
             bool ok = true;
             const int n1a = min(256, p.r_pad), n1b = p.r_pad - n1a;
             const uint32_t idesc_a = make_idesc_bf16(128, n1a, 0, 1);
             const uint32_t idesc_b = make_idesc_bf16(128, n1b > 0 ? n1b : 64, 0, 1);
-            for (int kb = 0; kb < nkb1 && ok; ++kb, ++it) {
-                const int s = it % NS;
-                ok = mbar_wait(smem_u32(&ctl->full[s]), (it / NS) & 1, abort_flag, p.status);
+            const uint64_t a_ring = make_smem_desc(ring, 16, 1024);                    // K-major tile at a stage start
+            const uint64_t b1_ring = make_smem_desc(ring + kTileBytes, 8192, 1024);   // MN-major B1 tile of a stage
+            for (int kb = 0; kb < nkb1; ++kb) {
+                ok = mbar_wait(full0 + 8 * rp.s, rp.ph, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_addr = ring + s * S;
-                const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
-                const uint64_t b_desc = make_smem_desc(a_addr + kTileBytes, 8192, 1024);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint32_t acc = (kb > 0 || kk > 0) ? 1u : 0u;
-                    tc_mma_bf16(tmem, desc_advance(a_desc, kk * 32), desc_advance(b_desc, kk * 2048), idesc_a, acc);
-                    if (n1b > 0)
-                        tc_mma_bf16(tmem + 256, desc_advance(a_desc, kk * 32),
-                                    desc_advance(b_desc, 4 * 8192 + kk * 2048), idesc_b, acc);
+                const uint64_t a_desc = a_ring + (rp.off >> 4), b_desc = b1_ring + (rp.off >> 4);
+                const uint32_t acc0 = kb > 0 ? 1u : 0u;
+                tc_mma_bf16(tmem, a_desc, b_desc, idesc_a, acc0);
+                tc_mma_bf16(tmem, a_desc + 2, b_desc + 128, idesc_a, 1u);
+                tc_mma_bf16(tmem, a_desc + 4, b_desc + 256, idesc_a, 1u);
+                tc_mma_bf16(tmem, a_desc + 6, b_desc + 384, idesc_a, 1u);
+                if (n1b > 0) {
+                    const uint64_t b2 = b_desc + (4 * 8192 >> 4);
+                    tc_mma_bf16(tmem + 256, a_desc, b2, idesc_b, acc0);
+                    tc_mma_bf16(tmem + 256, a_desc + 2, b2 + 128, idesc_b, 1u);
+                    tc_mma_bf16(tmem + 256, a_desc + 4, b2 + 256, idesc_b, 1u);
+                    tc_mma_bf16(tmem + 256, a_desc + 6, b2 + 384, idesc_b, 1u);
                 }
-                tc_commit(smem_u32(&ctl->empty[s]));
+                tc_commit(empty0 + 8 * rp.s);
+                rp.advance(NS, S);
             }
             if (ok) tc_commit(smem_u32(&ctl->t_full));
             if (ok) ok = mbar_wait(smem_u32(&ctl->t_ready), 0, abort_flag, p.status);
@@ -173,25 +203,31 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 tma_store_commit();
             }
             const uint32_t idesc2 = make_idesc_bf16(128, 128, 0, 0);
+            const uint64_t t_desc = make_smem_desc(t_smem, 16, 1024);
+            const uint32_t accf0 = smem_u32(&ctl->acc_full[0]), acce0 = smem_u32(&ctl->acc_empty[0]);
             for (int j = 0; j < ntile && ok; ++j) {
-                const int b = j & 1;
-                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), ((j >> 1) & 1) ^ 1u, abort_flag, p.status);
+                const uint32_t b = static_cast<uint32_t>(j) & (kAccBufs - 1);
+                ok = mbar_wait(acce0 + 8 * b, ((static_cast<uint32_t>(j) / kAccBufs) & 1u) ^ 1u, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                for (int kb = 0; kb < nkb2; ++kb, ++it) {
-                    const int s = it % NS;
-                    ok = mbar_wait(smem_u32(&ctl->full[s]), (it / NS) & 1, abort_flag, p.status);
+                const uint32_t d_tmem = tmem + b * 128;
+                for (int kb = 0; kb < nkb2; kb += bps) {
+                    const int nb = min(bps, nkb2 - kb);
+                    ok = mbar_wait(full0 + 8 * rp.s, rp.ph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t a_desc = make_smem_desc(t_smem + kb * kTileBytes, 16, 1024);
-                    const uint64_t b_desc = make_smem_desc(ring + s * S, 16, 1024);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        tc_mma_bf16(tmem + b * 128, desc_advance(a_desc, kk * 32), desc_advance(b_desc, kk * 32),
-                                    idesc2, (kb > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&ctl->empty[s]));
+                    for (int q = 0; q < nb; ++q) {
+                        const uint64_t a_desc = t_desc + static_cast<uint32_t>((kb + q) * (kTileBytes >> 4));
+                        const uint64_t b_desc = a_ring + ((rp.off + q * kTileBytes) >> 4);
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc2, (kb + q) > 0 ? 1u : 0u);
+                        tc_mma_bf16(d_tmem, a_desc + 2, b_desc + 2, idesc2, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 4, b_desc + 4, idesc2, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 6, b_desc + 6, idesc2, 1u);
+                    }
+                    tc_commit(empty0 + 8 * rp.s);
+                    rp.advance(NS, S);
                 }
-                if (ok) tc_commit(smem_u32(&ctl->acc_full[b]));
+                if (ok) tc_commit(accf0 + 8 * b);
             }
             if (stash) tma_store_wait_read<0>();
         }
@@ -200,7 +236,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const uint32_t lane_base = tmem + (static_cast<uint32_t>(q * 32) << 16);
-        bool ok = mbar_wait(smem_u32(&ctl->t_full), 0, abort_flag, p.status);
+        bool ok = mbar_wait_warp(smem_u32(&ctl->t_full), 0, abort_flag, p.status);
         tc_fence_after();
         if (ok) {
             const uint32_t sw = static_cast<uint32_t>(row & 7);
@@ -219,40 +255,51 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(smem_u32(&ctl->t_ready));
 
-        const int pieces = p.r_pad / 64;   // 8 KB staging pieces in the idle B1 part of each stage
+        // Store staging: two 4 KB panels (32 rows x 64 columns) per warp, used alternately, either
+        // in a dedicated region or (large r) in the B1 part of ring stages, idle during phase 2.
+        uint32_t stg0, stg1;
+        if (p.staging_off) {
+            stg0 = smem_u32(smem + p.staging_off) + q * 8192;
+            stg1 = stg0 + 4096;
+        } else {
+            const int pieces = p.r_pad / 64;          // 8 KB pieces per stage
+            stg0 = ring + (q / pieces) * S + kTileBytes + (q % pieces) * 8192;
+            stg1 = stg0 + 4096;
+        }
+        const uint32_t sw = static_cast<uint32_t>(lane & 7);
         bool stored = false;
+        const int r0 = m0 + q * 32;
         for (int j = 0; j < ntile && ok; ++j) {
-            const int b = j & 1;
-            ok = mbar_wait(smem_u32(&ctl->acc_full[b]), (j >> 1) & 1, abort_flag, p.status);
+            const uint32_t b = static_cast<uint32_t>(j) & (kAccBufs - 1);
+            ok = mbar_wait_warp(smem_u32(&ctl->acc_full[b]), (static_cast<uint32_t>(j) / kAccBufs) & 1u, abort_flag,
+                                p.status);
             tc_fence_after();
             if (!ok) break;
-            const int wb = q * 2 + b;
-            const uint32_t stg = ring + (wb / pieces) * S + kTileBytes + (wb % pieces) * 8192;
-            if (lane == 0) tma_store_wait_read<1>();   // the store that used this buffer two tiles ago
-            __syncwarp();
-            const uint32_t sw = static_cast<uint32_t>(lane & 7);
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(lane_base + b * 128 + c * 32, v);
-                tmem_ld_wait();
-                const uint32_t prow = stg + (c >> 1) * 4096 + lane * 128;
-                const uint32_t cb = (c & 1) * 4;
+            // drain the accumulator in one go and hand the TMEM buffer back before converting
+            uint32_t v[4][32];
 #pragma unroll
-                for (int t = 0; t < 4; ++t) st_shared_v4(prow + (((cb + t) ^ sw) << 4), pack8(v + 8 * t));
-            }
+            for (int c = 0; c < 4; ++c) tmem_ld32(lane_base + b * 128 + c * 32, v[c]);
+            tmem_ld_wait();
             tc_fence_before();
-            fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(smem_u32(&ctl->acc_empty[b]));
-                const int n0 = (t_beg + j) * 128, r0 = m0 + q * 32;
-                if (r0 < p.M) {
-                    tma_store_2d(&tmOut, stg, n0, r0);
-                    if (n0 + 64 < p.N2) tma_store_2d(&tmOut, stg + 4096, n0 + 64, r0);
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+            const int n0 = (t_beg + j) * 128;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t stg = h ? stg1 : stg0;
+                if (lane == 0) tma_store_wait_read<1>();   // the store that last read this panel buffer
+                __syncwarp();
+                const uint32_t prow = stg + lane * 128;
+#pragma unroll
+                for (int t = 0; t < 8; ++t)
+                    st_shared_v4(prow + ((static_cast<uint32_t>(t) ^ sw) << 4), pack8(v[2 * h + (t >> 2)] + 8 * (t & 3)));
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (r0 < p.M && n0 + 64 * h < p.N2) tma_store_2d(&tmOut, stg, n0 + 64 * h, r0);
+                    tma_store_commit();
+                    stored = true;
                 }
-                tma_store_commit();
-                stored = true;
             }
         }
         if (lane == 0 && stored) tma_store_wait_read<0>();
@@ -272,10 +319,13 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
     const int64_t r_pad = (r + 63) / 64 * 64;
     if (r_pad > 384 || M > 0x7fffffff || K1 > 0x7fffffff || N2 > 0x7fffffff) return false;
     const int64_t stage = kTileBytes + r_pad * 128;
-    const int64_t budget = 227 * 1024 - 2048 - r_pad * 256;
+    // Small ranks: dedicated 32 KB store staging, and a whole B2 tile (r_pad / 64 boxes) per stage
+    // in phase 2.  Larger ranks: staging lives in the idle B1 part of the stages, one box per stage.
+    const bool dedicated = r_pad <= 128;
+    const int64_t budget = 227 * 1024 - 2048 - r_pad * 256 - (dedicated ? 32768 : 0);
     int64_t ns = budget / stage;
     if (ns > kMaxStages) ns = kMaxStages;
-    if (ns < 2 || ns * (r_pad / 64) < 8) return false;
+    if (ns < 2 || (!dedicated && ns * (r_pad / 64) < 4)) return false;
     const int64_t row_tiles = ceil_div(M, 128), nt = ceil_div(N2, 128);
     // Split N2 over blockIdx.y while that shortens the critical path of a CTA (each split repeats
     // phase 1, cost ~ K1; phase 2 costs ~ N2 / split) and the grid still fits one wave.
@@ -294,7 +344,9 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
     plan->nsplit = static_cast<int>(has_out ? best : 1);
     plan->tiles_per_split = has_out ? static_cast<int>(ceil_div(nt, best)) : 0;
     plan->nsplit = has_out ? static_cast<int>(ceil_div(nt, plan->tiles_per_split)) : 1;
-    plan->smem = static_cast<size_t>(2048 + r_pad * 256 + ns * stage);
+    plan->smem = static_cast<size_t>(2048 + r_pad * 256 + ns * stage + (dedicated ? 32768 : 0));
+    plan->boxes_per_stage = dedicated ? static_cast<int>(r_pad / 64) : 1;
+    plan->staging_off = dedicated ? static_cast<int>(1024 + r_pad * 256 + ns * stage) : 0;
     plan->row_tiles = static_cast<int>(row_tiles);
     return true;
 }
@@ -315,6 +367,7 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
     p.M = static_cast<int>(M); p.K1 = static_cast<int>(K1); p.N2 = static_cast<int>(N2);
     p.r_pad = plan.r_pad; p.num_stages = plan.num_stages; p.stage_bytes = plan.stage_bytes;
     p.tiles_per_split = plan.tiles_per_split; p.store_T = T != nullptr;
+    p.boxes_per_stage = plan.boxes_per_stage; p.staging_off = plan.staging_off;
     p.status = device_status_ptr();
     static bool configured[64] = {};
     int dev = 0;

@@ -61,6 +61,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 #pragma unroll 1
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(32);   // pollers share the SM's barrier unit with the arrivals they wait for
         if ((it & 255u) == 0u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycleLimit) break;
@@ -69,6 +70,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1u;
     if (status) atomicExch(status, kStatusTimeout);
     return false;
+}
+
+// The same wait for a whole (converged) warp: lane 0 polls and broadcasts the verdict, so the
+// barrier word is not hammered by 32 pollers and the warp leaves the wait converged (the
+// elect.sync that usually follows needs all 32 lanes).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               unsigned int* status) {
+    uint32_t ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 // ---------------------------------------------------------------- TMA
@@ -90,6 +101,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// Ask L2 to fetch one tile of a tensor (no shared-memory destination, no completion to wait for).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int c0, int c1) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1)
+                 : "memory");
+}
 // Shared -> global tile store (bulk async group); rows/columns outside the tensor are clipped.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
