@@ -30,7 +30,7 @@ namespace tc {
 namespace {
 
 constexpr int kMaxStages = 8;
-constexpr int kChainThreads = 192;
+constexpr int kChainThreads = 320;          // producer warp, MMA warp, 8 epilogue warps
 constexpr uint32_t kTileBytes = 16384;      // 128 rows x 64 bf16
 constexpr int kAccBufs = 4;                 // 4 x 128 TMEM columns of phase-2 accumulators
 
@@ -103,10 +103,10 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->t_full), 1);
-        mbar_init(smem_u32(&ctl->t_ready), 4);
+        mbar_init(smem_u32(&ctl->t_ready), 8);
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
-            mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), 8);
         }
         ctl->abort = 0;
         fence_barrier_init();
@@ -233,14 +233,17 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
+        // Eight warps: warp w may touch the TMEM lanes of quadrant w % 4, so two warps share each
+        // 32-row quadrant and split the columns (64 of every 128) between them.
         const int q = warp & 3;
+        const int hcol = (warp - 2) >> 2;            // 0 or 1: which 64-column half of a tile
         const int row = q * 32 + lane;
         const uint32_t lane_base = tmem + (static_cast<uint32_t>(q * 32) << 16);
         bool ok = mbar_wait_warp(smem_u32(&ctl->t_full), 0, abort_flag, p.status);
         tc_fence_after();
+        const uint32_t sw = static_cast<uint32_t>(lane & 7);      // == row & 7
         if (ok) {
-            const uint32_t sw = static_cast<uint32_t>(row & 7);
-            for (int c = 0; c < p.r_pad / 32; ++c) {
+            for (int c = hcol; c < p.r_pad / 32; c += 2) {
                 uint32_t v[32];
                 tmem_ld32(lane_base + c * 32, v);
                 tmem_ld_wait();
@@ -255,48 +258,46 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(smem_u32(&ctl->t_ready));
 
-        // Store staging: two 4 KB panels (32 rows x 64 columns) per warp, used alternately, either
-        // in a dedicated region or (large r) in the B1 part of ring stages, idle during phase 2.
-        uint32_t stg0, stg1;
+        // Store staging: one 4 KB panel (32 rows x 64 columns) per warp, either in a dedicated
+        // region or (large r) in the B1 part of ring stages, which is idle during phase 2.
+        const int ew = warp - 2;                      // 0..7
+        uint32_t stg;
         if (p.staging_off) {
-            stg0 = smem_u32(smem + p.staging_off) + q * 8192;
-            stg1 = stg0 + 4096;
+            stg = smem_u32(smem + p.staging_off) + ew * 4096;
         } else {
-            const int pieces = p.r_pad / 64;          // 8 KB pieces per stage
-            stg0 = ring + (q / pieces) * S + kTileBytes + (q % pieces) * 8192;
-            stg1 = stg0 + 4096;
+            const int per_stage = p.r_pad / 32;       // 4 KB pieces in the B1 part of one stage
+            stg = ring + (ew / per_stage) * S + kTileBytes + (ew % per_stage) * 4096;
         }
-        const uint32_t sw = static_cast<uint32_t>(lane & 7);
         bool stored = false;
         const int r0 = m0 + q * 32;
+        const uint32_t prow = stg + lane * 128;
         for (int j = 0; j < ntile && ok; ++j) {
             const uint32_t b = static_cast<uint32_t>(j) & (kAccBufs - 1);
             ok = mbar_wait_warp(smem_u32(&ctl->acc_full[b]), (static_cast<uint32_t>(j) / kAccBufs) & 1u, abort_flag,
                                 p.status);
             tc_fence_after();
             if (!ok) break;
-            // drain the accumulator in one go and hand the TMEM buffer back before converting
-            uint32_t v[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(lane_base + b * 128 + c * 32, v[c]);
+            // drain this warp's 64 columns and hand the TMEM buffer back before converting
+            uint32_t v[2][32];
+            tmem_ld32(lane_base + b * 128 + hcol * 64, v[0]);
+            tmem_ld32(lane_base + b * 128 + hcol * 64 + 32, v[1]);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
-            const int n0 = (t_beg + j) * 128;
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                tma_store_wait_read<0>();             // the previous store has finished reading the panel
+            }
+            __syncwarp();
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint32_t stg = h ? stg1 : stg0;
-                if (lane == 0) tma_store_wait_read<1>();   // the store that last read this panel buffer
-                __syncwarp();
-                const uint32_t prow = stg + lane * 128;
-#pragma unroll
-                for (int t = 0; t < 8; ++t)
-                    st_shared_v4(prow + ((static_cast<uint32_t>(t) ^ sw) << 4), pack8(v[2 * h + (t >> 2)] + 8 * (t & 3)));
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    if (r0 < p.M && n0 + 64 * h < p.N2) tma_store_2d(&tmOut, stg, n0 + 64 * h, r0);
+            for (int t = 0; t < 8; ++t)
+                st_shared_v4(prow + ((static_cast<uint32_t>(t) ^ sw) << 4), pack8(v[t >> 2] + 8 * (t & 3)));
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                const int n0 = (t_beg + j) * 128 + hcol * 64;
+                if (r0 < p.M && n0 < p.N2) {
+                    tma_store_2d(&tmOut, stg, n0, r0);
                     tma_store_commit();
                     stored = true;
                 }
@@ -325,7 +326,7 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
     const int64_t budget = 227 * 1024 - 2048 - r_pad * 256 - (dedicated ? 32768 : 0);
     int64_t ns = budget / stage;
     if (ns > kMaxStages) ns = kMaxStages;
-    if (ns < 2 || (!dedicated && ns * (r_pad / 64) < 4)) return false;
+    if (ns < 2 || (!dedicated && ns * (r_pad / 32) < 8)) return false;
     const int64_t row_tiles = ceil_div(M, 128), nt = ceil_div(N2, 128);
     // Split N2 over blockIdx.y while that shortens the critical path of a CTA (each split repeats
     // phase 1, cost ~ K1; phase 2 costs ~ N2 / split) and the grid still fits one wave.

@@ -61,7 +61,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 #pragma unroll 1
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(32);   // pollers share the SM's barrier unit with the arrivals they wait for
         if ((it & 255u) == 0u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycleLimit) break;
