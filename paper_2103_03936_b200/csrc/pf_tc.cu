@@ -249,8 +249,8 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
     const int bn = pick_bn(N);
     CUtensorMap ta, tb;
-    const bool oka = A.mn_major ? make_map_2d(&ta, A.p, K, M, A.ld, 64) : make_map_2d(&ta, A.p, M, K, A.ld, kBM);
-    const bool okb = B.mn_major ? make_map_2d(&tb, B.p, K, N, B.ld, 64) : make_map_2d(&tb, B.p, N, K, B.ld, bn);
+    const bool oka = A.mn_major ? cached_map_2d(&ta, A.p, K, M, A.ld, 64) : cached_map_2d(&ta, A.p, M, K, A.ld, kBM);
+    const bool okb = B.mn_major ? cached_map_2d(&tb, B.p, K, N, B.ld, 64) : cached_map_2d(&tb, B.p, N, K, B.ld, bn);
     if (!oka || !okb) return PF_ERR_CUDA;
     GemmParams p;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);

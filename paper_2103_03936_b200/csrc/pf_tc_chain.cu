@@ -359,10 +359,10 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
     ChainPlan plan;
     if (!chain_plan(M, K1, N2, r, out != nullptr, &plan)) return PF_ERR_UNSUPPORTED;
     CUtensorMap ta, tb1, tb2, to, tt;
-    bool ok = make_map_2d(&ta, A, M, K1, lda, 128) && make_map_2d(&tb1, B1, K1, r, ldb1, 64) &&
-              make_map_2d(&tb2, B2, N2, r, ldb2, 128);
-    ok = ok && (out ? make_map_2d(&to, out, M, N2, ldo, 32) : make_map_2d(&to, A, M, K1, lda, 32));
-    ok = ok && (T ? make_map_2d(&tt, T, M, r, ldt, 128) : make_map_2d(&tt, A, M, K1, lda, 128));
+    bool ok = cached_map_2d(&ta, A, M, K1, lda, 128) && cached_map_2d(&tb1, B1, K1, r, ldb1, 64) &&
+              cached_map_2d(&tb2, B2, N2, r, ldb2, 128);
+    ok = ok && (out ? cached_map_2d(&to, out, M, N2, ldo, 32) : cached_map_2d(&to, A, M, K1, lda, 32));
+    ok = ok && (T ? cached_map_2d(&tt, T, M, r, ldt, 128) : cached_map_2d(&tt, A, M, K1, lda, 128));
     if (!ok) return PF_ERR_CUDA;
     ChainParams p;
     p.M = static_cast<int>(M); p.K1 = static_cast<int>(K1); p.N2 = static_cast<int>(N2);
