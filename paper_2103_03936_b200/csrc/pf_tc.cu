@@ -245,7 +245,7 @@ int pick_bn(int64_t N) { return N <= 64 ? 64 : 128; }
 
 // C[M,N] (bf16, ldc) = A * B.  `partial` must hold splits*M*N floats when splits > 1.
 int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
-         int splits, float* partial, cudaStream_t stream) {
+         int splits, float* partial, cudaStream_t stream, int* deferred_splits = nullptr) {
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
     const int bn = pick_bn(N);
     CUtensorMap ta, tb;
@@ -265,6 +265,10 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
     cudaError_t e = bn == 64 ? launch_gemm<64>(ta, tb, p, grid, stream) : launch_gemm<128>(ta, tb, p, grid, stream);
     if (e != cudaSuccess) return PF_ERR_CUDA;
+    if (deferred_splits) {           // the caller sums the slices (together with another product's)
+        *deferred_splits = p.splits;
+        return PF_OK;
+    }
     if (p.splits > 1) {
         e = splitk_reduce(partial, C, ldc, M, N, p.splits, PF_BF16, stream);
         if (e != cudaSuccess) return PF_ERR_CUDA;
@@ -400,6 +404,22 @@ int linear_bwd(const LinearArgs& a, int* handled) {
             st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
             if (st != PF_OK) return st;
         }
+    }
+    if (su > 1 && sv > 1) {
+        // both factor gradients are split over m: one launch sums the slices of both
+        int used_u = 0, used_v = 0;
+        st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream, &used_u);
+        if (st != PF_OK) return st;
+        st = gemm({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, a.stream, &used_v);
+        if (st != PF_OK) return st;
+        if (used_u > 1 && used_v > 1)
+            return splitk_reduce2_bf16(pu, a.dU, a.lddu, a.k, a.r, used_u, pv, a.dV, a.lddv, a.n, a.r, used_v,
+                                       a.stream) == cudaSuccess ? PF_OK : PF_ERR_CUDA;
+        if (used_u > 1 && splitk_reduce(pu, a.dU, a.lddu, a.k, a.r, used_u, PF_BF16, a.stream) != cudaSuccess)
+            return PF_ERR_CUDA;
+        if (used_v > 1 && splitk_reduce(pv, a.dV, a.lddv, a.n, a.r, used_v, PF_BF16, a.stream) != cudaSuccess)
+            return PF_ERR_CUDA;
+        return PF_OK;
     }
     st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream);
     if (st != PF_OK) return st;
