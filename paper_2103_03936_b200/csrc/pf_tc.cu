@@ -41,6 +41,12 @@ struct GemmParams {
     long long ldc;
     float* partial;          // fp32 [splits, M, N] when splits > 1
     unsigned int* status;
+    // Implicit-GEMM convolution operand A (tmA is then a 4-D NHWC map):
+    //   conv_mode 1 (dX): A K-major; row tile = cv_box_h full-width image rows of dT; k-block =
+    //                     (tap, 64-rank block), tap offsets flipped; B rows are offset by tap * cv_C.
+    //   conv_mode 2 (dU): A MN-major; row tile = (tap, 128-channel block) of the unrolled factor;
+    //                     k-block = 64 pixels (cv_box_h full-width rows) of the image x.
+    int conv_mode, cv_blks, cv_kw, cv_pad, cv_C, cv_box_h, cv_tpi;
 };
 
 __device__ __forceinline__ void store_row_chunk_bf16(__nv_bfloat16* dst, const uint32_t (&v)[32], int ncols,
@@ -127,7 +133,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint32_t b_dst = a_dst + kABytes;
                 mbar_expect_tx(full, kStageBytes);
                 const int k0 = (kb_beg + i) * kBK;
-                if (p.a_mn) {
+                if (p.conv_mode == 1) {
+                    const int kbg = kb_beg + i;
+                    const int tap = kbg / p.cv_blks, rb = kbg - tap * p.cv_blks;
+                    const int ta = tap / p.cv_kw, tb = tap - ta * p.cv_kw;
+                    const int img = static_cast<int>(blockIdx.x) / p.cv_tpi;
+                    const int h0 = (static_cast<int>(blockIdx.x) - img * p.cv_tpi) * p.cv_box_h;
+                    tma_load_4d(a_dst, &tmA, full, rb * 64, p.cv_pad - tb, h0 + p.cv_pad - ta, img);
+                    tma_load_2d(b_dst, &tmB, full, rb * 64, tap * p.cv_C + n0);
+                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                    continue;
+                }
+                if (p.conv_mode == 2) {
+                    const int kbg = kb_beg + i;
+                    const int tap = m0 / p.cv_C, c0 = m0 - tap * p.cv_C;
+                    const int ta = tap / p.cv_kw, tb = tap - ta * p.cv_kw;
+                    const int img = kbg / p.cv_tpi;
+                    const int h0 = (kbg - img * p.cv_tpi) * p.cv_box_h;
+                    tma_load_4d(a_dst, &tmA, full, c0, tb - p.cv_pad, h0 + ta - p.cv_pad, img);
+                    tma_load_4d(a_dst + 8192, &tmA, full, c0 + 64, tb - p.cv_pad, h0 + ta - p.cv_pad, img);
+                } else if (p.a_mn) {
                     tma_load_2d(a_dst, &tmA, full, m0, k0);
                     tma_load_2d(a_dst + 8192, &tmA, full, m0 + 64, k0);
                 } else {
@@ -244,13 +269,29 @@ int pick_splits(int64_t M, int64_t N, int bn, int64_t K) {
 int pick_bn(int64_t N) { return N <= 64 ? 64 : 128; }
 
 // C[M,N] (bf16, ldc) = A * B.  `partial` must hold splits*M*N floats when splits > 1.
+struct ConvA {
+    int mode;                   // 1: dX (A = dT image), 2: dU (A = x image)
+    int N, H, W, Cimg;          // the NHWC tensor A is read from (Cimg channels)
+    int kw, pad, Cw;            // kernel width, padding, channels of the layer input (rows per tap of U)
+};
+
 int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
-         int splits, float* partial, cudaStream_t stream, int* deferred_splits = nullptr) {
+         int splits, float* partial, cudaStream_t stream, int* deferred_splits = nullptr,
+         const ConvA* cv = nullptr) {
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
     const int bn = pick_bn(N);
     CUtensorMap ta, tb;
-    const bool oka = A.mn_major ? cached_map_2d(&ta, A.p, K, M, A.ld, 64) : cached_map_2d(&ta, A.p, M, K, A.ld, kBM);
-    const bool okb = B.mn_major ? cached_map_2d(&tb, B.p, K, N, B.ld, 64) : cached_map_2d(&tb, B.p, N, K, B.ld, bn);
+    bool oka, okb;
+    if (cv && cv->mode == 1) {          // B = U as a (taps * Cw) x R matrix, K-major
+        oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, 128 / cv->W);
+        okb = cached_map_2d(&tb, B.p, static_cast<int64_t>(K / cv->Cimg) * cv->Cw, cv->Cimg, B.ld, bn);
+    } else if (cv && cv->mode == 2) {
+        oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, 64 / cv->W);
+        okb = cached_map_2d(&tb, B.p, K, N, B.ld, 64);
+    } else {
+        oka = A.mn_major ? cached_map_2d(&ta, A.p, K, M, A.ld, 64) : cached_map_2d(&ta, A.p, M, K, A.ld, kBM);
+        okb = B.mn_major ? cached_map_2d(&tb, B.p, K, N, B.ld, 64) : cached_map_2d(&tb, B.p, N, K, B.ld, bn);
+    }
     if (!oka || !okb) return PF_ERR_CUDA;
     GemmParams p;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
@@ -259,6 +300,13 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     p.kb_per_split = static_cast<int>(ceil_div(nkb, splits));
     p.splits = static_cast<int>(ceil_div(nkb, p.kb_per_split));   // every slice gets >= 1 k-block
     p.C = C; p.ldc = ldc; p.partial = partial;
+    p.conv_mode = 0; p.cv_blks = 1; p.cv_kw = 1; p.cv_pad = 0; p.cv_C = 1; p.cv_box_h = 1; p.cv_tpi = 1;
+    if (cv) {
+        p.conv_mode = cv->mode; p.cv_kw = cv->kw; p.cv_pad = cv->pad; p.cv_C = cv->Cw;
+        p.cv_blks = cv->Cimg / 64;
+        p.cv_box_h = (cv->mode == 1 ? 128 : 64) / cv->W;
+        p.cv_tpi = cv->H / p.cv_box_h;
+    }
     p.status = device_status_ptr();
     dim3 grid(static_cast<unsigned>(ceil_div(M, kBM)), static_cast<unsigned>(ceil_div(N, bn)),
               static_cast<unsigned>(p.splits));
@@ -321,8 +369,6 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
     }
     return b;
 }
-
-size_t conv_extra_workspace(int, int, int, int, int, int, int, int, int, int, bool) { return 0; }
 
 int linear_fwd(const LinearArgs& a, int* handled) {
     *handled = 0;
@@ -426,8 +472,88 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     return gemm({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, a.stream);
 }
 
-int conv_fwd(const ConvArgs&, int* handled) { *handled = 0; return PF_OK; }
-int conv_bwd(const ConvArgs&, int* handled) { *handled = 0; return PF_OK; }
+// Tensor-core envelope of the factorized convolution: stride 1, "same" padding, channel counts
+// that tile evenly, image rows that pack into 128-pixel (forward, dX) and 64-pixel (dU) tiles.
+static bool conv_tc_ok(const ConvArgs& a) {
+    if (a.stride != 1 || a.kh != a.kw || 2 * a.pad != a.kh - 1) return false;
+    if (a.C % 128 != 0 || a.R % 64 != 0 || a.O % 8 != 0 || a.R > 384) return false;
+    if (a.W > 64 || 64 % a.W != 0 || a.H % (128 / a.W) != 0) return false;
+    if (static_cast<int64_t>(a.N) * a.H * a.W > 0x7fffffff) return false;
+    return encode_fn() != nullptr;
+}
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride, int pad,
+                            bool bwd) {
+    if (!bwd) return 0;
+    // split partials of dU ((kh*kw*C) x R) and dV (O x R)
+    const int64_t P = static_cast<int64_t>(N) * H * W, Keff = static_cast<int64_t>(kh) * kw * C;
+    const int su = pick_splits(Keff, R, pick_bn(R), P), sv = pick_splits(O, R, pick_bn(R), P);
+    (void)stride; (void)pad;
+    return align_up(su > 1 ? static_cast<size_t>(su) * Keff * R * 4 : 0, 256) +
+           align_up(sv > 1 ? static_cast<size_t>(sv) * O * R * 4 : 0, 256);
+}
+
+int conv_fwd(const ConvArgs& a, int* handled) {
+    *handled = 0;
+    if (!conv_tc_ok(a) || !aligned16(a.x) || !aligned16(a.U) || !aligned16(a.V) || !aligned16(a.y) ||
+        (a.T && !aligned16(a.T)))
+        return PF_OK;
+    const int64_t M = static_cast<int64_t>(a.N) * a.H * a.W, Keff = static_cast<int64_t>(a.kh) * a.kw * a.C;
+    ChainPlan plan;
+    if (!chain_plan(M, Keff, a.O, a.R, true, &plan)) return PF_OK;
+    *handled = 1;
+    const ChainConv cv{a.N, a.H, a.W, a.C, a.kh, a.kw, a.pad};
+    return chain(a.x, a.C, M, Keff, a.U, a.R, a.R, a.V, a.R, a.O, a.y, a.O, a.T, a.R, a.stream, &cv);
+}
+
+int conv_bwd(const ConvArgs& a, int* handled) {
+    *handled = 0;
+    if (!conv_tc_ok(a) || !aligned16(a.x) || !aligned16(a.U) || !aligned16(a.V) || !aligned16(a.dY) ||
+        (a.T && !aligned16(a.T)) || (a.dX && !aligned16(a.dX)))
+        return PF_OK;
+    const int64_t M = static_cast<int64_t>(a.N) * a.H * a.W, Keff = static_cast<int64_t>(a.kh) * a.kw * a.C;
+    ChainPlan plan;
+    if (!a.T && !chain_plan(M, Keff, a.O, a.R, false, &plan)) return PF_OK;
+    *handled = 1;
+    int st;
+    const void* T = a.T;
+    if (!T) {   // recompute the thin convolution (phase 1 of the forward only)
+        const ChainConv cv{a.N, a.H, a.W, a.C, a.kh, a.kw, a.pad};
+        st = chain(a.x, a.C, M, Keff, a.U, a.R, a.R, a.V, a.R, a.O, nullptr, a.O, a.ws_T, a.R, a.stream, &cv);
+        if (st != PF_OK) return st;
+        T = a.ws_T;
+    }
+    void* dT = a.ws_G;
+    const int su = pick_splits(Keff, a.R, pick_bn(a.R), M), sv = pick_splits(a.O, a.R, pick_bn(a.R), M);
+    float* pu = reinterpret_cast<float*>(a.ws);
+    float* pv = reinterpret_cast<float*>(a.ws + align_up(su > 1 ? static_cast<size_t>(su) * Keff * a.R * 4 : 0, 256));
+    // dT = dY V  (per pixel)
+    st = gemm({a.dY, a.O, false}, {a.V, a.R, true}, M, a.R, a.O, dT, a.R, 1, nullptr, a.stream);
+    if (st != PF_OK) return st;
+    // dX = sum over taps of shifted dT times U[tap]^T  (implicit GEMM, contraction kh*kw*R)
+    if (a.dX) {
+        const ConvA cx{1, a.N, a.H, a.W, a.R, a.kw, a.pad, a.C};
+        st = gemm({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
+                  nullptr, a.stream, nullptr, &cx);
+        if (st != PF_OK) return st;
+    }
+    // dU[tap] = shifted x^T dT ; dV = dY^T T   (reductions over all pixels, split across CTAs)
+    int used_u = 0, used_v = 0;
+    const ConvA cu{2, a.N, a.H, a.W, a.C, a.kw, a.pad, a.C};
+    st = gemm({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, a.stream, &used_u, &cu);
+    if (st != PF_OK) return st;
+    st = gemm({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, a.stream, &used_v);
+    if (st != PF_OK) return st;
+    if (used_u > 1 && used_v > 1)
+        return splitk_reduce2_bf16(pu, a.dU, a.R, Keff, a.R, used_u, pv, a.dV, a.R, a.O, a.R, used_v, a.stream) ==
+                       cudaSuccess ? PF_OK : PF_ERR_CUDA;
+    if (used_u > 1 && splitk_reduce(pu, a.dU, a.R, Keff, a.R, used_u, PF_BF16, a.stream) != cudaSuccess)
+        return PF_ERR_CUDA;
+    if (used_v > 1 && splitk_reduce(pv, a.dV, a.R, a.O, a.R, used_v, PF_BF16, a.stream) != cudaSuccess)
+        return PF_ERR_CUDA;
+    return PF_OK;
+}
 
 }  // namespace tc
 }  // namespace pf

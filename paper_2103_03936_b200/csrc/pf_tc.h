@@ -35,9 +35,14 @@ struct ChainPlan {
     size_t smem;
 };
 bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan);
+// When `conv` is given, A is an NHWC image and phase 1 is the implicit GEMM of a kh x kw, stride-1,
+// "same"-padded convolution: M = N*H*W pixels, K1 = kh*kw*C, B1 = U as a (kh*kw*C) x r matrix.
+struct ChainConv {
+    int N, H, W, C, kh, kw, pad;
+};
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
-          cudaStream_t stream);
+          cudaStream_t stream, const ChainConv* conv = nullptr);
 
 size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool bwd);
 size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,

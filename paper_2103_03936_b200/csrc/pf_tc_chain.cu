@@ -54,6 +54,9 @@ struct ChainParams {
     int store_T;
     int boxes_per_stage;    // phase 2: B2 boxes (16 KB each) loaded per ring stage
     int staging_off;        // byte offset (from the 1 KB-aligned base) of dedicated store staging, 0 = none
+    // Implicit-GEMM convolution as phase 1 (conv_cblks > 0): tmA is a 4-D NHWC map, a row tile is
+    // box_h full-width image rows (box_h * W = 128 pixels) and k-block kb = (tap, 64-channel block).
+    int conv_cblks, conv_kw, conv_pad, conv_box_h, conv_tiles_per_img;
     unsigned int* status;
 };
 
@@ -145,7 +148,15 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const uint32_t full = full0 + 8 * rp.s;
                 const uint32_t dst = ring + rp.off;
                 mbar_expect_tx(full, tx1);
-                tma_load_2d(dst, &tmA, full, kb * 64, m0);
+                if (p.conv_cblks > 0) {
+                    const int tap = kb / p.conv_cblks, cb = kb - tap * p.conv_cblks;
+                    const int ta = tap / p.conv_kw, tb = tap - ta * p.conv_kw;
+                    const int img = static_cast<int>(blockIdx.x) / p.conv_tiles_per_img;
+                    const int h0 = (static_cast<int>(blockIdx.x) - img * p.conv_tiles_per_img) * p.conv_box_h;
+                    tma_load_4d(dst, &tmA, full, cb * 64, tb - p.conv_pad, h0 + ta - p.conv_pad, img);
+                } else {
+                    tma_load_2d(dst, &tmA, full, kb * 64, m0);
+                }
                 for (int q = 0; q < nkb2; ++q)
                     tma_load_2d(dst + kTileBytes + q * 8192, &tmB1, full, q * 64, kb * 64);
                 rp.advance(NS, S);
@@ -355,20 +366,26 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
 // out may be null (phase 1 only: T is written and nothing else).  All pointers must satisfy tma_ok.
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
-          cudaStream_t stream) {
+          cudaStream_t stream, const ChainConv* conv) {
     ChainPlan plan;
     if (!chain_plan(M, K1, N2, r, out != nullptr, &plan)) return PF_ERR_UNSUPPORTED;
     CUtensorMap ta, tb1, tb2, to, tt;
-    bool ok = cached_map_2d(&ta, A, M, K1, lda, 128) && cached_map_2d(&tb1, B1, K1, r, ldb1, 64) &&
-              cached_map_2d(&tb2, B2, N2, r, ldb2, 128);
-    ok = ok && (out ? cached_map_2d(&to, out, M, N2, ldo, 32) : cached_map_2d(&to, A, M, K1, lda, 32));
-    ok = ok && (T ? cached_map_2d(&tt, T, M, r, ldt, 128) : cached_map_2d(&tt, A, M, K1, lda, 128));
+    bool ok = conv ? cached_map_nhwc(&ta, A, conv->N, conv->H, conv->W, conv->C, conv->W, 128 / conv->W)
+                   : cached_map_2d(&ta, A, M, K1, lda, 128);
+    ok = ok && cached_map_2d(&tb1, B1, K1, r, ldb1, 64) && cached_map_2d(&tb2, B2, N2, r, ldb2, 128);
+    ok = ok && (out ? cached_map_2d(&to, out, M, N2, ldo, 32) : cached_map_2d(&to, B2, N2, r, ldb2, 32));
+    ok = ok && (T ? cached_map_2d(&tt, T, M, r, ldt, 128) : cached_map_2d(&tt, B2, N2, r, ldb2, 128));
     if (!ok) return PF_ERR_CUDA;
     ChainParams p;
     p.M = static_cast<int>(M); p.K1 = static_cast<int>(K1); p.N2 = static_cast<int>(N2);
     p.r_pad = plan.r_pad; p.num_stages = plan.num_stages; p.stage_bytes = plan.stage_bytes;
     p.tiles_per_split = plan.tiles_per_split; p.store_T = T != nullptr;
     p.boxes_per_stage = plan.boxes_per_stage; p.staging_off = plan.staging_off;
+    p.conv_cblks = 0; p.conv_kw = 1; p.conv_pad = 0; p.conv_box_h = 1; p.conv_tiles_per_img = 1;
+    if (conv) {
+        p.conv_cblks = conv->C / 64; p.conv_kw = conv->kw; p.conv_pad = conv->pad;
+        p.conv_box_h = 128 / conv->W; p.conv_tiles_per_img = conv->H / p.conv_box_h;
+    }
     p.status = device_status_ptr();
     static bool configured[64] = {};
     int dev = 0;

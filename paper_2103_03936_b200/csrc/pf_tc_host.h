@@ -71,6 +71,37 @@ inline bool cached_map_2d(CUtensorMap* map, const void* p, int64_t rows, int64_t
     return true;
 }
 
+// 4-D bf16 tensor map over an NHWC image [N, H, W, C]: boxes are 64 channels x box_w x box_h pixels
+// of one image (box_w * box_h rows of 128 bytes in shared memory, pixel-major); coordinates may
+// start outside the image (zero padding of the convolution), out-of-range pixels read as zero.
+inline bool cached_map_nhwc(CUtensorMap* map, const void* p, int64_t N, int64_t H, int64_t W, int64_t C,
+                            int box_w, int box_h) {
+    constexpr int kSlots = 64;
+    struct Slot { MapKey key; CUtensorMap map; bool used; };
+    static Slot slots[kSlots];
+    static std::mutex mu;
+    const MapKey key{p, N * 100003 + H, C, W, -(box_h * 1024 + box_w)};
+    const uint64_t h = reinterpret_cast<uintptr_t>(p) * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(key.rows) * 31 +
+                       static_cast<uint64_t>(C) * 131 + static_cast<uint64_t>(W) * 1031 + static_cast<uint64_t>(-key.box_rows);
+    Slot& s = slots[(h >> 20) % kSlots];
+    std::lock_guard<std::mutex> lock(mu);
+    if (s.used && s.key == key) { *map = s.map; return true; }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
+                                static_cast<cuuint64_t>(N)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 2, static_cast<cuuint64_t>(W) * C * 2,
+                                   static_cast<cuuint64_t>(H) * W * C * 2};
+    const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(box_w), static_cast<cuuint32_t>(box_h), 1u};
+    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(p), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    s.key = key; s.map = *map; s.used = true;
+    return true;
+}
+
 inline bool tma_ok(const void* p, int64_t ld) {
     return (reinterpret_cast<uintptr_t>(p) & 15) == 0 && (ld % 8) == 0 && ld * 2 < (1LL << 40);
 }

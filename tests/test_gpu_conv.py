@@ -71,6 +71,17 @@ def test_multi_tile(dtype, N, H, W, C, R, O):
     run_conv(wl.ConvCase("mt", N, H, W, C, R, O, dtype, 60))
 
 
+@pytest.mark.parametrize("N,H,W,C,R,O,k", [(2, 32, 32, 128, 64, 128, 3), (3, 16, 16, 256, 64, 64, 3),
+                                           (2, 16, 32, 128, 64, 96, 3), (1, 64, 64, 128, 64, 128, 3),
+                                           (2, 32, 32, 128, 128, 256, 5), (2, 8, 16, 128, 192, 64, 1)])
+def test_tensor_core_envelope(N, H, W, C, R, O, k):
+    """Shapes inside the implicit-GEMM tensor-core envelope (stride 1, 'same' padding, C % 128 == 0,
+    R % 64 == 0, image rows packing into 128- and 64-pixel tiles), with and without stash / dX."""
+    run_conv(wl.ConvCase("tc", N, H, W, C, R, O, wl.BF16, 63, kh=k, kw=k, pad=(k - 1) // 2))
+    run_conv(wl.ConvCase("tc", N, H, W, C, R, O, wl.BF16, 64, kh=k, kw=k, pad=(k - 1) // 2), stash=False,
+             need_dX=False)
+
+
 def test_recompute_without_stash_and_no_dX():
     run_conv(wl.ConvCase("ns", 2, 16, 16, 64, 16, 64, wl.BF16, 61), stash=False)
     run_conv(wl.ConvCase("nx", 2, 16, 16, 64, 16, 64, wl.BF16, 62), need_dX=False)
