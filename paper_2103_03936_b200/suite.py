@@ -1,0 +1,187 @@
+"""Per-configuration timings of the factorized layers (forward, backward, fraction of roofline).
+
+Used by ``bench.py --suite FILE``: every benchmark configuration (tiny fp32, Transformer FFN,
+LSTM gates in the tight and in a 16-byte-pitch layout, ResNet-style convolutions with the gradient
+pack, and the rank sweep) is timed with CUDA events on rotating buffer sets larger than L2, and
+written as one JSON object per line.  Only timing lives here; parity is the tests' job.
+"""
+from __future__ import annotations
+
+import json
+import math
+
+import torch
+
+import pf_workloads as wl
+from . import binding as pf
+
+L2_BYTES = 126 << 20
+
+
+def _rand(shape, dtype, scale=1.0, relu=False, ld=None):
+    rows = int(math.prod(shape[:-1]))
+    cols = shape[-1]
+    if ld is None:
+        t = torch.randn(shape, device="cuda", dtype=torch.float32) * scale
+        if relu:
+            t = t.clamp_(min=0)
+        return t.to(dtype)
+    buf = torch.zeros((rows, ld), device="cuda", dtype=dtype)
+    buf[:, :cols] = (torch.randn((rows, cols), device="cuda", dtype=torch.float32) * scale).to(dtype)
+    return buf[:, :cols]
+
+
+def _time(calls_per_set, iters, warmup=3):
+    """calls_per_set: list (one per buffer set) of (fwd_call, bwd_call[, extra_call])."""
+    ns = len(calls_per_set)
+    for i in range(warmup):
+        for c in calls_per_set[i % ns]:
+            c()
+    torch.cuda.synchronize()
+    evs = []
+    for i in range(iters):
+        cs = calls_per_set[i % ns]
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(len(cs) + 1)]
+        e[0].record()
+        for j, c in enumerate(cs):
+            c()
+            e[j + 1].record()
+        evs.append(e)
+    torch.cuda.synchronize()
+    out = []
+    for j in range(len(calls_per_set[0])):
+        ts = sorted(e[j].elapsed_time(e[j + 1]) * 1e3 for e in evs)
+        out.append({"median_us": ts[len(ts) // 2], "min_us": ts[0]})
+    return out
+
+
+def _floors(flops_fwd, bytes_fwd, bytes_bwd, pk):
+    f = max(flops_fwd / (pk["bf16_tflops"] * 1e12), bytes_fwd / (pk["hbm_gbs"] * 1e9)) * 1e6
+    b = max(2 * flops_fwd / (pk["bf16_tflops"] * 1e12), bytes_bwd / (pk["hbm_gbs"] * 1e9)) * 1e6
+    return f, b
+
+
+def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=30):
+    tdt = torch.bfloat16 if dtype == wl.BF16 else torch.float32
+    s = 2 if dtype == wl.BF16 else 4
+    code = pf.PF_BF16 if dtype == wl.BF16 else pf.PF_F32
+    foot = s * (2 * m * k + 2 * m * n + m * r)
+    nsets = max(1, min(16, math.ceil(4 * L2_BYTES / foot)))
+    ldk = (k + 7) // 8 * 8 if pad_pitch else None
+    ldr = (r + 7) // 8 * 8 if pad_pitch else None
+    sig = 1.0 / math.sqrt(k)
+    U, V = _rand((k, r), tdt, sig, ld=ldr), _rand((n, r), tdt, sig, ld=ldr)
+    stream = torch.cuda.current_stream()
+    sets = []
+    for _ in range(nsets):
+        x, dY = _rand((m, k), tdt, ld=ldk), _rand((m, n), tdt)
+        y = torch.empty((m, n), dtype=tdt, device="cuda")
+        T = _rand((m, r), tdt, ld=ldr)
+        dX = _rand((m, k), tdt, ld=ldk)
+        dU, dV = _rand((k, r), tdt, ld=ldr), _rand((n, r), tdt, ld=ldr)
+        wf = torch.empty(max(256, pf.pf_lowrank_linear_workspace(m, k, n, r, code, 0)), dtype=torch.uint8, device="cuda")
+        wb = torch.empty(max(256, pf.pf_lowrank_linear_workspace(m, k, n, r, code, 1)), dtype=torch.uint8, device="cuda")
+        f, _ = pf.pf_lowrank_linear_fwd(x, U, V, y=y, T_stash=T, workspace=wf, stream=stream, prepare=True)
+        b, _ = pf.pf_lowrank_linear_bwd(x, U, V, dY, T_stash=T, dX=dX, dU=dU, dV=dV, workspace=wb, stream=stream,
+                                        prepare=True)
+        sets.append((f, b))
+    l0 = pf.pf_launch_count()
+    for c in sets[0]:
+        c()
+    launches = pf.pf_launch_count() - l0
+    t = _time(sets, iters)
+    flops_fwd = 2.0 * m * r * (k + n)
+    bytes_fwd = s * (m * k + m * n + r * (k + n))
+    bytes_bwd = s * (m * n + 2 * m * k + 2 * r * (k + n))
+    ff, fb = _floors(flops_fwd, bytes_fwd, bytes_bwd, pk)
+    tot = t[0]["median_us"] + t[1]["median_us"]
+    return {"config": name, "kind": "linear", "m": m, "k": k, "n": n, "r": r, "dtype": dtype,
+            "pitch": "padded to 16 B" if pad_pitch else "tight", "buffer_sets": nsets, "launches_fwd_bwd": launches,
+            "fwd_us": t[0]["median_us"], "bwd_us": t[1]["median_us"], "fwd_bwd_us": tot,
+            "floor_fwd_us": ff, "floor_bwd_us": fb, "roofline_frac": (ff + fb) / tot,
+            "tflops": 3 * flops_fwd / tot / 1e6, "gbs": (bytes_fwd + bytes_bwd) / tot / 1e3}
+
+
+def conv_config(name, c, pk, iters=20):
+    tdt = torch.bfloat16
+    M = c.N * c.H * c.W
+    foot = 2 * (2 * M * c.C + 2 * M * c.O + M * c.R)
+    nsets = max(1, min(8, math.ceil(4 * L2_BYTES / foot)))
+    U = _rand((c.kh, c.kw, c.C, c.R), tdt, math.sqrt(2.0 / (c.kh * c.kw * c.C)))
+    V = _rand((c.O, c.R), tdt, math.sqrt(2.0 / c.R))
+    stream = torch.cuda.current_stream()
+    sets = []
+    for _ in range(nsets):
+        x = _rand((c.N, c.H, c.W, c.C), tdt, relu=True)
+        dY = _rand((c.N, c.H, c.W, c.O), tdt)
+        y = torch.empty_like(dY)
+        T = torch.empty((c.N, c.H, c.W, c.R), dtype=tdt, device="cuda")
+        dX, dU, dV = torch.empty_like(x), torch.empty_like(U), torch.empty_like(V)
+        args = (c.N, c.H, c.W, c.C, c.R, c.O, c.kh, c.kw, c.stride, c.pad, pf.PF_BF16)
+        wf = torch.empty(max(256, pf.pf_lowrank_conv_workspace(*args, 0)), dtype=torch.uint8, device="cuda")
+        wb = torch.empty(max(256, pf.pf_lowrank_conv_workspace(*args, 1)), dtype=torch.uint8, device="cuda")
+        f, _ = pf.pf_lowrank_conv_fwd(x, U, V, stride=c.stride, pad=c.pad, y=y, T_stash=T, workspace=wf,
+                                      stream=stream, prepare=True)
+        b, _ = pf.pf_lowrank_conv_bwd(x, U, V, dY, stride=c.stride, pad=c.pad, T_stash=T, dX=dX, dU=dU, dV=dV,
+                                      workspace=wb, stream=stream, prepare=True)
+        flat = torch.empty(dU.numel() + dV.numel(), dtype=tdt, device="cuda")
+        pk_call, _ = pf.pf_pack_factor_grads([dU, dV], flat=flat, stream=stream, prepare=True)
+        sets.append((f, b, pk_call))
+    l0 = pf.pf_launch_count()
+    for cc in sets[0]:
+        cc()
+    launches = pf.pf_launch_count() - l0
+    t = _time(sets, iters)
+    Keff = c.kh * c.kw * c.C
+    flops_fwd = 2.0 * M * c.R * (Keff + c.O)
+    bytes_fwd = 2 * (M * c.C + M * c.O + c.R * (Keff + c.O))
+    bytes_bwd = 2 * (M * c.O + 2 * M * c.C + 2 * c.R * (Keff + c.O))
+    ff, fb = _floors(flops_fwd, bytes_fwd, bytes_bwd, pk)
+    tot = t[0]["median_us"] + t[1]["median_us"]
+    return {"config": name, "kind": "conv", "N": c.N, "H": c.H, "W": c.W, "C": c.C, "R": c.R, "O": c.O,
+            "dtype": "bf16", "buffer_sets": nsets, "launches_fwd_bwd_pack": launches,
+            "fwd_us": t[0]["median_us"], "bwd_us": t[1]["median_us"], "pack_us": t[2]["median_us"],
+            "fwd_bwd_us": tot, "floor_fwd_us": ff, "floor_bwd_us": fb, "roofline_frac": (ff + fb) / tot,
+            "tflops": 3 * flops_fwd / tot / 1e6, "gbs": (bytes_fwd + bytes_bwd) / tot / 1e3}
+
+
+def pack_config(name, numels, pk, iters=30):
+    tdt = torch.bfloat16
+    grads = [torch.randn(n, device="cuda").to(tdt) for n in numels]
+    total = sum(numels)
+    nsets = max(1, min(8, math.ceil(2 * L2_BYTES / (4 * total))))
+    stream = torch.cuda.current_stream()
+    sets = []
+    for _ in range(nsets):
+        g = [t.clone() for t in grads]
+        flat = torch.empty(total, dtype=tdt, device="cuda")
+        call, _ = pf.pf_pack_factor_grads(g, flat=flat, stream=stream, prepare=True)
+        sets.append((call,))
+    t = _time(sets, iters)
+    us = t[0]["median_us"]
+    return {"config": name, "kind": "pack", "tensors": len(numels), "elements": total, "dtype": "bf16",
+            "us": us, "gbs": 4.0 * total / us / 1e3, "roofline_frac": (4.0 * total / (pk["hbm_gbs"] * 1e9) * 1e6) / us}
+
+
+def run(path, pk):
+    rows = []
+
+    def emit(r):
+        rows.append(r)
+        with open(path, "w") as f:
+            for rr in rows:
+                f.write(json.dumps(rr) + "\n")
+
+    emit(linear_config("C1 tiny fp32", 64, 256, 256, 32, wl.F32, pk))
+    emit(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk))
+    emit(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk))
+    emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk))
+    emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True))
+    for name, c in wl.conv_cases().items():
+        emit(conv_config(f"{name} conv", c, pk))
+    for r in wl.SWEEP_RANKS:
+        emit(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=12))
+    # ResNet-18-sized and Transformer-sized factor-gradient lists (Table 4 / Table 3 parameter counts)
+    emit(pack_config("pack ~3.3M elements", [147457, 16384, 589821, 65536, 1179653, 131072, 1179648, 131071], pk))
+    emit(pack_config("pack ~26.7M elements", [65536 + (i % 3) for i in range(100)] + [262144 - (i % 5) for i in range(76)], pk))
+    return rows
