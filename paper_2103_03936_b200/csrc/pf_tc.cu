@@ -12,6 +12,8 @@
 
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "pf_tc_host.h"
 #include "pf_tc_prims.cuh"
 
@@ -260,6 +262,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
 int pick_splits(int64_t M, int64_t N, int bn, int64_t K) {
     const int64_t tiles = ceil_div(M, kBM) * ceil_div(N, bn);
     const int64_t nkb = ceil_div(K, kBK);
+    if (tiles < 1 || nkb < 1) return 1;
     int64_t s = kNumSMs / tiles;
     if (s > nkb / 4) s = nkb / 4;     // at least 4 k-blocks per slice
     if (s > 64) s = 64;
@@ -367,6 +370,9 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
         const size_t pv = sv > 1 ? static_cast<size_t>(sv) * n * r * 4 : 0;
         b += align_up(pu, 256) + align_up(pv, 256);
     }
+    // skinny batches: the m x r products (x U, dY V) are split over their contraction to fill the SMs
+    const int s1 = std::max(pick_splits(m, r, pick_bn(r), k), bwd ? pick_splits(m, r, pick_bn(r), n) : 1);
+    b += align_up(s1 > 1 ? static_cast<size_t>(s1) * m * r * 4 : 0, 256);
     return b;
 }
 
@@ -392,7 +398,9 @@ int linear_fwd(const LinearArgs& a, int* handled) {
         st = chain(x.p, x.ld, a.m, a.k, U.p, U.ld, a.r, V.p, V.ld, a.n, a.y, a.ldy, a.T ? T : nullptr, ldT,
                    a.stream);
     } else {
-        st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, T, ldT, 1, nullptr, a.stream);
+        float* p1 = reinterpret_cast<float*>(scratch + align_up(static_cast<size_t>(a.m) * pad8(a.r) * 2, 256));
+        st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, T, ldT,
+                  pick_splits(a.m, a.r, pick_bn(a.r), a.k), p1, a.stream);
         if (st != PF_OK) return st;
         st = gemm({T, ldT, false}, {V.p, V.ld, false}, a.m, a.n, a.r, a.y, a.ldy, 1, nullptr, a.stream);
     }
@@ -426,9 +434,9 @@ int linear_bwd(const LinearArgs& a, int* handled) {
         }
     }
     *handled = 1;
+    bool need_T = false;
     if (!a.T) {
-        st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, Tbuf, pad8(a.r), 1, nullptr, a.stream);
-        if (st != PF_OK) return st;
+        need_T = true;
         T.p = Tbuf; T.ld = pad8(a.r);
     }
     char* G = scratch;
@@ -438,13 +446,21 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     float* pu = reinterpret_cast<float*>(scratch);
     scratch += align_up(su > 1 ? static_cast<size_t>(su) * a.k * a.r * 4 : 0, 256);
     float* pv = reinterpret_cast<float*>(scratch);
+    scratch += align_up(sv > 1 ? static_cast<size_t>(sv) * a.n * a.r * 4 : 0, 256);
+    float* p1 = reinterpret_cast<float*>(scratch);
     // G = dY V ; dX = G U^T ; dU = x^T G ; dV = dY^T T
+    if (need_T) {   // no stash: recompute T = x U
+        st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, Tbuf, pad8(a.r),
+                  pick_splits(a.m, a.r, pick_bn(a.r), a.k), p1, a.stream);
+        if (st != PF_OK) return st;
+    }
     ChainPlan plan;
     if (use_chain(a.m) && (!a.dX || tma_ok(a.dX, a.lddx)) && chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan)) {
         st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream);
         if (st != PF_OK) return st;
     } else {
-        st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG, 1, nullptr, a.stream);
+        st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG,
+                  pick_splits(a.m, a.r, pick_bn(a.r), a.n), p1, a.stream);
         if (st != PF_OK) return st;
         if (a.dX) {
             st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
