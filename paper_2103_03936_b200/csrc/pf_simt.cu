@@ -166,10 +166,16 @@ splitk_reduce2_kernel(const ReduceJob a, const ReduceJob b, int blocks_a) {
     const int64_t slice4 = total4;
     const float4* src = reinterpret_cast<const float4*>(j.partial);
     for (int64_t e = blk * blockDim.x + threadIdx.x; e < total4; e += nblk * blockDim.x) {
-        float4 acc = __ldcs(src + e);
-        for (int z = 1; z < j.splits; ++z) {
-            const float4 t = __ldcs(src + z * slice4 + e);
-            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        // slices are summed in increasing order; loads are issued eight at a time so that the
+        // memory latency is paid once per batch, not once per slice
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int z0 = 0; z0 < j.splits; z0 += 8) {
+            float4 t[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                t[u] = (z0 + u < j.splits) ? __ldcs(src + (z0 + u) * slice4 + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
         }
         const int64_t el = e * 4, row = el / j.N, col = el - row * j.N;
         __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);

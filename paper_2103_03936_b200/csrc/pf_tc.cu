@@ -121,6 +121,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();                 // everything above overlapped the previous kernel's tail
+    pdl_launch_dependents();
     const uint32_t tmem_base = ctl->tmem_base;
 
     // Producer and MMA issuer are each one thread chosen with elect.sync that runs its whole role
@@ -253,8 +255,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Gemm
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    tc_gemm_kernel<BN><<<grid, kGemmThreads, smem, stream>>>(ta, tb, p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_overlapped(tc_gemm_kernel<BN>, grid, dim3(kGemmThreads), smem, stream, ta, tb, p);
     if (e == cudaSuccess) count_launch();
     return e;
 }

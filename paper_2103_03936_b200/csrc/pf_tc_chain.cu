@@ -123,6 +123,8 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();                 // everything above overlapped the previous kernel's tail
+    pdl_launch_dependents();
     const uint32_t tmem = ctl->tmem_base;
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
 
@@ -397,8 +399,9 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
         configured[dev] = true;
     }
     dim3 grid(static_cast<unsigned>(plan.row_tiles), static_cast<unsigned>(plan.nsplit), 1);
-    tc_chain_kernel<<<grid, kChainThreads, plan.smem, stream>>>(ta, tb1, tb2, to, tt, p);
-    if (cudaGetLastError() != cudaSuccess) return PF_ERR_CUDA;
+    if (launch_overlapped(tc_chain_kernel, grid, dim3(kChainThreads), plan.smem, stream, ta, tb1, tb2, to, tt, p) !=
+        cudaSuccess)
+        return PF_ERR_CUDA;
     count_launch();
     return PF_OK;
 }

@@ -8,6 +8,7 @@
 #include <stdint.h>
 
 #include <mutex>
+#include <utility>
 
 namespace pf {
 namespace tc {
@@ -100,6 +101,21 @@ inline bool cached_map_nhwc(CUtensorMap* map, const void* p, int64_t N, int64_t 
         return false;
     s.key = key; s.map = *map; s.used = true;
     return true;
+}
+
+// Launch with programmatic stream serialization: the kernel's prologue (barrier set-up, TMEM
+// allocation, descriptor prefetch) overlaps the tail of the previous kernel in the stream; the
+// kernel itself calls griddepcontrol.wait before it touches global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 inline bool tma_ok(const void* p, int64_t ld) {
