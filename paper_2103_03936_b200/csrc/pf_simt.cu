@@ -158,24 +158,36 @@ struct ReduceJob {
 };
 __global__ void __launch_bounds__(256)
 splitk_reduce2_kernel(const ReduceJob a, const ReduceJob b, int blocks_a) {
+    // A block sums 64 consecutive float4 elements; its four 64-thread groups each take every
+    // fourth slice (in increasing order) and the four group sums are then added in group order,
+    // so the association is fixed and the result is bit-reproducible run to run.
+    __shared__ float4 part[3][64];
     const bool first = static_cast<int>(blockIdx.x) < blocks_a;
     const ReduceJob& j = first ? a : b;
-    const int64_t nblk = first ? blocks_a : static_cast<int>(gridDim.x) - blocks_a;
     const int64_t blk = first ? blockIdx.x : blockIdx.x - blocks_a;
     const int64_t total4 = j.M * j.N / 4;           // N % 4 == 0 on this path
-    const int64_t slice4 = total4;
+    const int lane64 = threadIdx.x & 63, grp = threadIdx.x >> 6;
+    const int64_t e = blk * 64 + lane64;
     const float4* src = reinterpret_cast<const float4*>(j.partial);
-    for (int64_t e = blk * blockDim.x + threadIdx.x; e < total4; e += nblk * blockDim.x) {
-        // slices are summed in increasing order; loads are issued eight at a time so that the
-        // memory latency is paid once per batch, not once per slice
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int z0 = 0; z0 < j.splits; z0 += 8) {
-            float4 t[8];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (e < total4) {
+        for (int z0 = grp; z0 < j.splits; z0 += 16) {
+            float4 t[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-                t[u] = (z0 + u < j.splits) ? __ldcs(src + (z0 + u) * slice4 + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int u = 0; u < 4; ++u)
+                t[u] = (z0 + 4 * u < j.splits) ? __ldcs(src + static_cast<int64_t>(z0 + 4 * u) * total4 + e)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
+            for (int u = 0; u < 4; ++u) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
+        }
+    }
+    if (grp > 0) part[grp - 1][lane64] = acc;
+    __syncthreads();
+    if (grp == 0 && e < total4) {
+#pragma unroll
+        for (int g = 0; g < 3; ++g) {
+            const float4 t = part[g][lane64];
+            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
         }
         const int64_t el = e * 4, row = el / j.N, col = el - row * j.N;
         __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
@@ -261,10 +273,8 @@ cudaError_t splitk_reduce2_bf16(const float* pa, void* Ca, int64_t ldca, int64_t
         return splitk_reduce(pb, Cb, ldcb, Mb, Nb, sb, PF_BF16, stream);
     }
     const ReduceJob a{pa, Ca, ldca, Ma, Na, sa}, b{pb, Cb, ldcb, Mb, Nb, sb};
-    auto blocks = [](int64_t M, int64_t N) {
-        int64_t n = ceil_div(M * N / 4, 256);
-        return static_cast<int>(n < 1 ? 1 : (n > 2 * kNumSMs ? 2 * kNumSMs : n));
-    };
+    auto blocks = [](int64_t M, int64_t N) { return static_cast<int>(ceil_div(M * N / 4, 64)); };
+    if (ceil_div(Ma * Na / 4, 64) + ceil_div(Mb * Nb / 4, 64) > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     const int ba = blocks(Ma, Na), bb = blocks(Mb, Nb);
     splitk_reduce2_kernel<<<ba + bb, 256, 0, stream>>>(a, b, ba);
     cudaError_t e = cudaGetLastError();
