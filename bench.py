@@ -358,7 +358,7 @@ def run_ours(args):
             from paper_2103_03936_b200 import suite
             del w
             torch.cuda.empty_cache()
-            suite.run(args.suite, pk)
+            suite.run(args.suite, pk, only=args.suite_only)
         print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
@@ -371,6 +371,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--suite", default=None, help="also write per-config timings to this file")
+    ap.add_argument("--suite-only", default=None, help="substring filter on suite configuration names")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

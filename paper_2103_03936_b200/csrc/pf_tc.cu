@@ -283,7 +283,8 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
          int splits, float* partial, cudaStream_t stream, int* deferred_splits = nullptr,
          const ConvA* cv = nullptr) {
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
-    const int bn = pick_bn(N);
+    // wide outputs that would need more than one wave of 128-column tiles take 256-column tiles
+    const int bn = (splits <= 1 && N >= 512 && ceil_div(M, kBM) * ceil_div(N, 128) > kNumSMs) ? 256 : pick_bn(N);
     CUtensorMap ta, tb;
     bool oka, okb;
     if (cv && cv->mode == 1) {          // B = U as a (taps * Cw) x R matrix, K-major
@@ -315,7 +316,9 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     dim3 grid(static_cast<unsigned>(ceil_div(M, kBM)), static_cast<unsigned>(ceil_div(N, bn)),
               static_cast<unsigned>(p.splits));
     if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
-    cudaError_t e = bn == 64 ? launch_gemm<64>(ta, tb, p, grid, stream) : launch_gemm<128>(ta, tb, p, grid, stream);
+    cudaError_t e = bn == 64    ? launch_gemm<64>(ta, tb, p, grid, stream)
+                    : bn == 128 ? launch_gemm<128>(ta, tb, p, grid, stream)
+                                : launch_gemm<256>(ta, tb, p, grid, stream);
     if (e != cudaSuccess) return PF_ERR_CUDA;
     if (deferred_splits) {           // the caller sums the slices (together with another product's)
         *deferred_splits = p.splits;

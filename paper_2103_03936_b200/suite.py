@@ -163,25 +163,38 @@ def pack_config(name, numels, pk, iters=30):
             "us": us, "gbs": 4.0 * total / us / 1e3, "roofline_frac": (4.0 * total / (pk["hbm_gbs"] * 1e9) * 1e6) / us}
 
 
-def run(path, pk):
+def run(path, pk, only=None):
+    """only: optional substring; configurations whose name lacks it are skipped."""
     rows = []
 
     def emit(r):
+        if r is None:
+            return
         rows.append(r)
         with open(path, "w") as f:
             for rr in rows:
                 f.write(json.dumps(rr) + "\n")
 
-    emit(linear_config("C1 tiny fp32", 64, 256, 256, 32, wl.F32, pk))
-    emit(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk))
-    emit(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk))
-    emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk))
-    emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True))
+    want = (lambda nm: only is None or only in nm)
+    if want("C1 tiny fp32"):
+        emit(linear_config("C1 tiny fp32", 64, 256, 256, 32, wl.F32, pk))
+    if want("C2a FFN up"):
+        emit(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk))
+    if want("C2b FFN down"):
+        emit(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk))
+    if want("C3 LSTM gates"):
+        emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk))
+    if want("C3 LSTM gates"):
+        emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True))
     for name, c in wl.conv_cases().items():
-        emit(conv_config(f"{name} conv", c, pk))
+        if want(f"{name} conv"):
+            emit(conv_config(f"{name} conv", c, pk))
     for r in wl.SWEEP_RANKS:
-        emit(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=12))
+        if want(f"C5 sweep r={r}"):
+            emit(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=12))
     # ResNet-18-sized and Transformer-sized factor-gradient lists (Table 4 / Table 3 parameter counts)
-    emit(pack_config("pack ~3.3M elements", [147457, 16384, 589821, 65536, 1179653, 131072, 1179648, 131071], pk))
-    emit(pack_config("pack ~26.7M elements", [65536 + (i % 3) for i in range(100)] + [262144 - (i % 5) for i in range(76)], pk))
+    if want("pack ~3.3M elements"):
+        emit(pack_config("pack ~3.3M elements", [147457, 16384, 589821, 65536, 1179653, 131072, 1179648, 131071], pk))
+    if want("pack ~26.7M elements"):
+        emit(pack_config("pack ~26.7M elements", [65536 + (i % 3) for i in range(100)] + [262144 - (i % 5) for i in range(76)], pk))
     return rows
