@@ -49,6 +49,9 @@ struct GemmParams {
     //   conv_mode 2 (dU): A MN-major; row tile = (tap, 128-channel block) of the unrolled factor;
     //                     k-block = 64 pixels (cv_box_h full-width rows) of the image x.
     int conv_mode, cv_blks, cv_kw, cv_pad, cv_C, cv_box_h, cv_tpi;
+    int rows_tile;           // output rows per CTA: 128, or cv_box_h * W pixels for conv_mode 1
+    int kpix;                // conv_mode 2: pixels per k-block (cv_box_h * W <= 64), else 64
+    int nkb_total;           // k-blocks of the whole contraction
 };
 
 __device__ __forceinline__ void store_row_chunk_bf16(__nv_bfloat16* dst, const uint32_t (&v)[32], int ncols,
@@ -99,8 +102,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile uint32_t* abort_flag = &ctl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * BN;
-    const int nkb_total = (p.K + kBK - 1) / kBK;
+    const int m0 = blockIdx.x * p.rows_tile, n0 = blockIdx.y * BN;
+    const int nkb_total = p.nkb_total;
     const int kb_beg = blockIdx.z * p.kb_per_split;
     const int kb_end = min(nkb_total, kb_beg + p.kb_per_split);
     const int nkb = kb_end - kb_beg;
@@ -116,6 +119,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         fence_proxy_async_smem();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
+    }
+    if (p.conv_mode == 2 && p.kpix < 64) {
+        // k-blocks hold fewer than 64 pixels: the unused contraction rows of every A stage must be
+        // zero (TMA never writes them), so that they add nothing to the sum
+        for (int i = threadIdx.x; i < kStages * static_cast<int>(kABytes / 16); i += blockDim.x) {
+            const int st = i / static_cast<int>(kABytes / 16), off = i - st * static_cast<int>(kABytes / 16);
+            *reinterpret_cast<uint4*>(tiles + st * kStageBytes + off * 16) = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async_smem();
     }
     if (warp == 1) tmem_alloc(smem_u32(&ctl->tmem_base), BN);
     tc_fence_before();
@@ -135,7 +147,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint32_t full = smem_u32(&ctl->full[s]);
                 const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
                 const uint32_t b_dst = a_dst + kABytes;
-                mbar_expect_tx(full, kStageBytes);
+                mbar_expect_tx(full, p.conv_mode == 1 ? static_cast<uint32_t>(p.rows_tile) * 128u + kBBytes
+                                     : p.conv_mode == 2 ? static_cast<uint32_t>(p.kpix) * 256u + kBBytes
+                                                        : kStageBytes);
                 const int k0 = (kb_beg + i) * kBK;
                 if (p.conv_mode == 1) {
                     const int kbg = kb_beg + i;
@@ -156,6 +170,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int h0 = (kbg - img * p.cv_tpi) * p.cv_box_h;
                     tma_load_4d(a_dst, &tmA, full, c0, tb - p.cv_pad, h0 + ta - p.cv_pad, img);
                     tma_load_4d(a_dst + 8192, &tmA, full, c0 + 64, tb - p.cv_pad, h0 + ta - p.cv_pad, img);
+#pragma unroll
+                    for (int h = 0; h < BN / 64; ++h) tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, kbg * p.kpix);
+                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                    continue;
                 } else if (p.a_mn) {
                     tma_load_2d(a_dst, &tmA, full, m0, k0);
                     tma_load_2d(a_dst + 8192, &tmA, full, m0 + 64, k0);
@@ -203,7 +221,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         if (ok) {
             const int row = m0 + q * 32 + lane;
-            const bool row_ok = row < p.M;
+            const bool row_ok = row < p.M && q * 32 + lane < p.rows_tile;
             __nv_bfloat16* crow = nullptr;
             float* prow = nullptr;
             bool vec_ok;
@@ -288,10 +306,10 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     CUtensorMap ta, tb;
     bool oka, okb;
     if (cv && cv->mode == 1) {          // B = U as a (taps * Cw) x R matrix, K-major
-        oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, 128 / cv->W);
+        oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, conv_box_h(cv->H, cv->W, 128));
         okb = cached_map_2d(&tb, B.p, static_cast<int64_t>(K / cv->Cimg) * cv->Cw, cv->Cimg, B.ld, bn);
     } else if (cv && cv->mode == 2) {
-        oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, 64 / cv->W);
+        oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, conv_box_h(cv->H, cv->W, 64));
         okb = cached_map_2d(&tb, B.p, K, N, B.ld, 64);
     } else {
         oka = A.mn_major ? cached_map_2d(&ta, A.p, K, M, A.ld, 64) : cached_map_2d(&ta, A.p, M, K, A.ld, kBM);
@@ -301,19 +319,22 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     GemmParams p;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.a_mn = A.mn_major; p.b_mn = B.mn_major;
-    const int64_t nkb = ceil_div(K, kBK);
-    p.kb_per_split = static_cast<int>(ceil_div(nkb, splits));
-    p.splits = static_cast<int>(ceil_div(nkb, p.kb_per_split));   // every slice gets >= 1 k-block
     p.C = C; p.ldc = ldc; p.partial = partial;
     p.conv_mode = 0; p.cv_blks = 1; p.cv_kw = 1; p.cv_pad = 0; p.cv_C = 1; p.cv_box_h = 1; p.cv_tpi = 1;
     if (cv) {
         p.conv_mode = cv->mode; p.cv_kw = cv->kw; p.cv_pad = cv->pad; p.cv_C = cv->Cw;
         p.cv_blks = cv->Cimg / 64;
-        p.cv_box_h = (cv->mode == 1 ? 128 : 64) / cv->W;
+        p.cv_box_h = conv_box_h(cv->H, cv->W, cv->mode == 1 ? 128 : 64);
         p.cv_tpi = cv->H / p.cv_box_h;
     }
+    p.rows_tile = (cv && cv->mode == 1) ? p.cv_box_h * cv->W : kBM;
+    p.kpix = (cv && cv->mode == 2) ? p.cv_box_h * cv->W : kBK;
+    const int64_t nkb = ceil_div(K, p.kpix);
+    p.nkb_total = static_cast<int>(nkb);
+    p.kb_per_split = static_cast<int>(ceil_div(nkb, splits < 1 ? 1 : splits));
+    p.splits = static_cast<int>(ceil_div(nkb, p.kb_per_split));   // every slice gets >= 1 k-block
     p.status = device_status_ptr();
-    dim3 grid(static_cast<unsigned>(ceil_div(M, kBM)), static_cast<unsigned>(ceil_div(N, bn)),
+    dim3 grid(static_cast<unsigned>(ceil_div(M, p.rows_tile)), static_cast<unsigned>(ceil_div(N, bn)),
               static_cast<unsigned>(p.splits));
     if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
     cudaError_t e = bn == 64    ? launch_gemm<64>(ta, tb, p, grid, stream)
@@ -497,7 +518,7 @@ int linear_bwd(const LinearArgs& a, int* handled) {
 static bool conv_tc_ok(const ConvArgs& a) {
     if (a.stride != 1 || a.kh != a.kw || 2 * a.pad != a.kh - 1) return false;
     if (a.C % 128 != 0 || a.R % 64 != 0 || a.O % 8 != 0 || a.R > 384) return false;
-    if (a.W > 64 || 64 % a.W != 0 || a.H % (128 / a.W) != 0) return false;
+    if (a.W > 64) return false;                       // one image row must fit a 64-pixel k-block of dU
     if (static_cast<int64_t>(a.N) * a.H * a.W > 0x7fffffff) return false;
     return encode_fn() != nullptr;
 }

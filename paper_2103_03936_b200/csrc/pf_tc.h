@@ -34,7 +34,8 @@ struct ChainPlan {
     int r_pad, num_stages, stage_bytes, nsplit, tiles_per_split, row_tiles, boxes_per_stage, staging_off;
     size_t smem;
 };
-bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan);
+bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan, int rows_tile = 128);
+int conv_box_h(int H, int W, int limit);
 // When `conv` is given, A is an NHWC image and phase 1 is the implicit GEMM of a kh x kw, stride-1,
 // "same"-padded convolution: M = N*H*W pixels, K1 = kh*kw*C, B1 = U as a (kh*kw*C) x r matrix.
 struct ChainConv {

@@ -57,6 +57,7 @@ struct ChainParams {
     // Implicit-GEMM convolution as phase 1 (conv_cblks > 0): tmA is a 4-D NHWC map, a row tile is
     // box_h full-width image rows (box_h * W = 128 pixels) and k-block kb = (tap, 64-channel block).
     int conv_cblks, conv_kw, conv_pad, conv_box_h, conv_tiles_per_img;
+    int rows_tile;          // rows of A one CTA owns: 128, or box_h * W pixels (<= 128) for the convolution
     unsigned int* status;
 };
 
@@ -90,7 +91,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     volatile uint32_t* abort_flag = &ctl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * 128;
+    const int m0 = blockIdx.x * p.rows_tile;
     const int nt_total = (p.N2 + 127) / 128;
     const int t_beg = blockIdx.y * p.tiles_per_split;
     const int ntile = max(0, min(nt_total, t_beg + p.tiles_per_split) - t_beg);
@@ -143,7 +144,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int n0 = (t_beg + static_cast<int>(blockIdx.x) % ntile) * 128;
                 for (int q = 0; q < nkb2; ++q) tma_prefetch_l2_2d(&tmB2, q * 64, n0);
             }
-            const uint32_t tx1 = kTileBytes + static_cast<uint32_t>(p.r_pad) * 128u;
+            const uint32_t tx1 = static_cast<uint32_t>(p.rows_tile) * 128u + static_cast<uint32_t>(p.r_pad) * 128u;
             for (int kb = 0; kb < nkb1; ++kb) {
                 ok = mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status);
                 if (!ok) break;
@@ -212,7 +213,10 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             tc_fence_after();
             const bool stash = ok && p.store_T && blockIdx.y == 0;
             if (stash) {
-                for (int q = 0; q < nkb2; ++q) tma_store_2d(&tmT, t_smem + q * kTileBytes, q * 64, m0);
+                for (int q = 0; q < nkb2; ++q) {
+                    if (p.conv_cblks > 0) tma_store_3d(&tmT, t_smem + q * kTileBytes, q * 64, 0, blockIdx.x);
+                    else tma_store_2d(&tmT, t_smem + q * kTileBytes, q * 64, m0);
+                }
                 tma_store_commit();
             }
             const uint32_t idesc2 = make_idesc_bf16(128, 128, 0, 0);
@@ -309,8 +313,9 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             __syncwarp();
             if (lane == 0) {
                 const int n0 = (t_beg + j) * 128 + hcol * 64;
-                if (r0 < p.M && n0 < p.N2) {
-                    tma_store_2d(&tmOut, stg, n0, r0);
+                if (r0 < p.M && q * 32 < p.rows_tile && n0 < p.N2) {
+                    if (p.conv_cblks > 0) tma_store_3d(&tmOut, stg, n0, q * 32, blockIdx.x);
+                    else tma_store_2d(&tmOut, stg, n0, r0);
                     tma_store_commit();
                     stored = true;
                 }
@@ -328,8 +333,16 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
 }  // namespace
 
+// Largest number of full-width image rows (a divisor of H) whose pixels fit in `limit` tile rows.
+int conv_box_h(int H, int W, int limit) {
+    int best = 1;
+    for (int d = 1; d <= H; ++d)
+        if (H % d == 0 && d * W <= limit) best = d;
+    return best;
+}
+
 // Shape envelope of the fused kernel and its launch geometry.
-bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan) {
+bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan, int rows_tile) {
     const int64_t r_pad = (r + 63) / 64 * 64;
     if (r_pad > 384 || M > 0x7fffffff || K1 > 0x7fffffff || N2 > 0x7fffffff) return false;
     const int64_t stage = kTileBytes + r_pad * 128;
@@ -340,7 +353,7 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
     int64_t ns = budget / stage;
     if (ns > kMaxStages) ns = kMaxStages;
     if (ns < 2 || (!dedicated && ns * (r_pad / 32) < 8)) return false;
-    const int64_t row_tiles = ceil_div(M, 128), nt = ceil_div(N2, 128);
+    const int64_t row_tiles = ceil_div(M, rows_tile), nt = ceil_div(N2, 128);
     // Split N2 over blockIdx.y while that shortens the critical path of a CTA (each split repeats
     // phase 1, cost ~ K1; phase 2 costs ~ N2 / split) and the grid still fits one wave.
     int64_t best = 1;
@@ -370,13 +383,22 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
           cudaStream_t stream, const ChainConv* conv) {
     ChainPlan plan;
-    if (!chain_plan(M, K1, N2, r, out != nullptr, &plan)) return PF_ERR_UNSUPPORTED;
+    const int box_h = conv ? conv_box_h(conv->H, conv->W, 128) : 1;
+    const int rows_tile = conv ? box_h * conv->W : 128;
+    if (!chain_plan(M, K1, N2, r, out != nullptr, &plan, rows_tile)) return PF_ERR_UNSUPPORTED;
     CUtensorMap ta, tb1, tb2, to, tt;
-    bool ok = conv ? cached_map_nhwc(&ta, A, conv->N, conv->H, conv->W, conv->C, conv->W, 128 / conv->W)
+    bool ok = conv ? cached_map_nhwc(&ta, A, conv->N, conv->H, conv->W, conv->C, conv->W, box_h)
                    : cached_map_2d(&ta, A, M, K1, lda, 128);
     ok = ok && cached_map_2d(&tb1, B1, K1, r, ldb1, 64) && cached_map_2d(&tb2, B2, N2, r, ldb2, 128);
-    ok = ok && (out ? cached_map_2d(&to, out, M, N2, ldo, 32) : cached_map_2d(&to, B2, N2, r, ldb2, 32));
-    ok = ok && (T ? cached_map_2d(&tt, T, M, r, ldt, 128) : cached_map_2d(&tt, B2, N2, r, ldb2, 128));
+    if (conv) {   // outputs seen as [tiles][rows_tile][cols] so that partial tiles are clipped per tile
+        ok = ok && (out ? cached_map_tiled_rows(&to, out, M / rows_tile, rows_tile, N2, 32)
+                        : cached_map_2d(&to, B2, N2, r, ldb2, 32));
+        ok = ok && (T ? cached_map_tiled_rows(&tt, T, M / rows_tile, rows_tile, r, rows_tile)
+                      : cached_map_2d(&tt, B2, N2, r, ldb2, 128));
+    } else {
+        ok = ok && (out ? cached_map_2d(&to, out, M, N2, ldo, 32) : cached_map_2d(&to, B2, N2, r, ldb2, 32));
+        ok = ok && (T ? cached_map_2d(&tt, T, M, r, ldt, 128) : cached_map_2d(&tt, B2, N2, r, ldb2, 128));
+    }
     if (!ok) return PF_ERR_CUDA;
     ChainParams p;
     p.M = static_cast<int>(M); p.K1 = static_cast<int>(K1); p.N2 = static_cast<int>(N2);
@@ -386,8 +408,9 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
     p.conv_cblks = 0; p.conv_kw = 1; p.conv_pad = 0; p.conv_box_h = 1; p.conv_tiles_per_img = 1;
     if (conv) {
         p.conv_cblks = conv->C / 64; p.conv_kw = conv->kw; p.conv_pad = conv->pad;
-        p.conv_box_h = 128 / conv->W; p.conv_tiles_per_img = conv->H / p.conv_box_h;
+        p.conv_box_h = box_h; p.conv_tiles_per_img = conv->H / box_h;
     }
+    p.rows_tile = rows_tile;
     p.status = device_status_ptr();
     static bool configured[64] = {};
     int dev = 0;

@@ -103,6 +103,37 @@ inline bool cached_map_nhwc(CUtensorMap* map, const void* p, int64_t N, int64_t 
     return true;
 }
 
+// 3-D view of a contiguous row-major [tiles * rows_tile, cols] matrix as [tiles][rows_tile][cols]:
+// a store box of box_rows rows that starts inside a tile is clipped at the end of that tile, which
+// is how partially filled 128-row MMA tiles (image rows that do not pack into 128 pixels) are
+// written without touching the next tile's pixels.
+inline bool cached_map_tiled_rows(CUtensorMap* map, const void* p, int64_t tiles, int rows_tile, int64_t cols,
+                                  int box_rows) {
+    constexpr int kSlots = 64;
+    struct Slot { MapKey key; CUtensorMap map; bool used; };
+    static Slot slots[kSlots];
+    static std::mutex mu;
+    const MapKey key{p, tiles, cols, rows_tile, -(1 << 24) - box_rows};
+    const uint64_t h = reinterpret_cast<uintptr_t>(p) * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(tiles) * 31 +
+                       static_cast<uint64_t>(cols) * 131 + static_cast<uint64_t>(rows_tile) * 1031 + box_rows;
+    Slot& s = slots[(h >> 20) % kSlots];
+    std::lock_guard<std::mutex> lock(mu);
+    if (s.used && s.key == key) { *map = s.map; return true; }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows_tile),
+                                static_cast<cuuint64_t>(tiles)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(cols) * 2, static_cast<cuuint64_t>(rows_tile) * cols * 2};
+    const cuuint32_t box[3] = {64u, static_cast<cuuint32_t>(box_rows), 1u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(p), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    s.key = key; s.map = *map; s.used = true;
+    return true;
+}
+
 // Launch with programmatic stream serialization: the kernel's prologue (barrier set-up, TMEM
 // allocation, descriptor prefetch) overlaps the tail of the previous kernel in the stream; the
 // kernel itself calls griddepcontrol.wait before it touches global memory.

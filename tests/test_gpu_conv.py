@@ -73,7 +73,10 @@ def test_multi_tile(dtype, N, H, W, C, R, O):
 
 @pytest.mark.parametrize("N,H,W,C,R,O,k", [(2, 32, 32, 128, 64, 128, 3), (3, 16, 16, 256, 64, 64, 3),
                                            (2, 16, 32, 128, 64, 96, 3), (1, 64, 64, 128, 64, 128, 3),
-                                           (2, 32, 32, 128, 128, 256, 5), (2, 8, 16, 128, 192, 64, 1)])
+                                           (2, 32, 32, 128, 128, 256, 5), (2, 8, 16, 128, 192, 64, 1),
+                                           (3, 14, 14, 128, 64, 128, 3), (2, 7, 7, 256, 64, 64, 3),
+                                           (2, 28, 28, 128, 64, 72, 3), (3, 10, 6, 128, 64, 64, 3),
+                                           (1, 3, 64, 128, 64, 64, 3)])
 def test_tensor_core_envelope(N, H, W, C, R, O, k):
     """Shapes inside the implicit-GEMM tensor-core envelope (stride 1, 'same' padding, C % 128 == 0,
     R % 64 == 0, image rows packing into 128- and 64-pixel tiles), with and without stash / dX."""
