@@ -88,9 +88,8 @@ __device__ __forceinline__ void store_row_chunk_f32(float* dst, const uint32_t (
 }
 
 template <int BN>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const GemmParams p) {
+__device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
+                                          const int bx, const int by, const int bz) {
     constexpr uint32_t kABytes = kBM * kBK * 2;          // 16 KB
     constexpr uint32_t kBBytes = BN * kBK * 2;
     constexpr uint32_t kStageBytes = kABytes + kBBytes;
@@ -102,9 +101,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile uint32_t* abort_flag = &ctl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * p.rows_tile, n0 = blockIdx.y * BN;
+    const int m0 = bx * p.rows_tile, n0 = by * BN;
     const int nkb_total = p.nkb_total;
-    const int kb_beg = blockIdx.z * p.kb_per_split;
+    const int kb_beg = bz * p.kb_per_split;
     const int kb_end = min(nkb_total, kb_beg + p.kb_per_split);
     const int nkb = kb_end - kb_beg;
 
@@ -155,8 +154,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int kbg = kb_beg + i;
                     const int tap = kbg / p.cv_blks, rb = kbg - tap * p.cv_blks;
                     const int ta = tap / p.cv_kw, tb = tap - ta * p.cv_kw;
-                    const int img = static_cast<int>(blockIdx.x) / p.cv_tpi;
-                    const int h0 = (static_cast<int>(blockIdx.x) - img * p.cv_tpi) * p.cv_box_h;
+                    const int img = bx / p.cv_tpi;
+                    const int h0 = (bx - img * p.cv_tpi) * p.cv_box_h;
                     tma_load_4d(a_dst, &tmA, full, rb * 64, p.cv_pad - tb, h0 + p.cv_pad - ta, img);
                     tma_load_2d(b_dst, &tmB, full, rb * 64, tap * p.cv_C + n0);
                     if (++s == kStages) { s = 0; ph ^= 1u; }
@@ -226,7 +225,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float* prow = nullptr;
             bool vec_ok;
             if (p.splits > 1) {
-                prow = p.partial + (static_cast<size_t>(blockIdx.z) * p.M + (row_ok ? row : 0)) * p.N;
+                prow = p.partial + (static_cast<size_t>(bz) * p.M + (row_ok ? row : 0)) * p.N;
                 vec_ok = (p.N % 4) == 0;
             } else {
                 crow = reinterpret_cast<__nv_bfloat16*>(p.C) + static_cast<size_t>(row_ok ? row : 0) * p.ldc;
@@ -249,6 +248,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, BN);
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const GemmParams p) {
+    gemm_tile<BN>(tmA, tmB, p, blockIdx.x, blockIdx.y, blockIdx.z);
+}
+
+// Two independent products in one launch (dU = x^T G and dV = dY^T T of one layer): CTAs
+// [0, ctas_a) work on problem a, the rest on problem b; each decodes (row tile, column tile, slice)
+// from its linear index.  One launch pays the start-up latency once and packs the short CTAs of
+// one problem into the tail of the other.
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
+                const GemmParams p0, const GemmParams p1, const int ctas_a, const int2 tiles_a, const int2 tiles_b) {
+    const bool first = static_cast<int>(blockIdx.x) < ctas_a;
+    const int idx = first ? blockIdx.x : blockIdx.x - ctas_a;
+    const int2 t = first ? tiles_a : tiles_b;             // (row tiles, column tiles)
+    const int bx = idx % t.x, by = (idx / t.x) % t.y, bz = idx / (t.x * t.y);
+    if (first) gemm_tile<BN>(tmA0, tmB0, p0, bx, by, bz);
+    else gemm_tile<BN>(tmA1, tmB1, p1, bx, by, bz);
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -297,13 +320,21 @@ struct ConvA {
     int kw, pad, Cw;            // kernel width, padding, channels of the layer input (rows per tap of U)
 };
 
-int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
-         int splits, float* partial, cudaStream_t stream, int* deferred_splits = nullptr,
-         const ConvA* cv = nullptr) {
+struct GemmLaunch {
+    CUtensorMap ta, tb;
+    GemmParams p;
+    dim3 grid;
+    int bn;
+};
+
+// Encodes the tensor maps and launch geometry of C[M,N] = A * B without launching.
+int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
+                 int splits, float* partial, const ConvA* cv, GemmLaunch* out) {
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
     // wide outputs that would need more than one wave of 128-column tiles take 256-column tiles
     const int bn = (splits <= 1 && N >= 512 && ceil_div(M, kBM) * ceil_div(N, 128) > kNumSMs) ? 256 : pick_bn(N);
-    CUtensorMap ta, tb;
+    CUtensorMap& ta = out->ta;
+    CUtensorMap& tb = out->tb;
     bool oka, okb;
     if (cv && cv->mode == 1) {          // B = U as a (taps * Cw) x R matrix, K-major
         oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, conv_box_h(cv->H, cv->W, 128));
@@ -316,7 +347,7 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
         okb = B.mn_major ? cached_map_2d(&tb, B.p, K, N, B.ld, 64) : cached_map_2d(&tb, B.p, N, K, B.ld, bn);
     }
     if (!oka || !okb) return PF_ERR_CUDA;
-    GemmParams p;
+    GemmParams& p = out->p;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.a_mn = A.mn_major; p.b_mn = B.mn_major;
     p.C = C; p.ldc = ldc; p.partial = partial;
@@ -337,9 +368,21 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     dim3 grid(static_cast<unsigned>(ceil_div(M, p.rows_tile)), static_cast<unsigned>(ceil_div(N, bn)),
               static_cast<unsigned>(p.splits));
     if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
-    cudaError_t e = bn == 64    ? launch_gemm<64>(ta, tb, p, grid, stream)
-                    : bn == 128 ? launch_gemm<128>(ta, tb, p, grid, stream)
-                                : launch_gemm<256>(ta, tb, p, grid, stream);
+    out->grid = grid;
+    out->bn = bn;
+    return PF_OK;
+}
+
+int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
+         int splits, float* partial, cudaStream_t stream, int* deferred_splits = nullptr,
+         const ConvA* cv = nullptr) {
+    GemmLaunch g;
+    const int st = gemm_prepare(A, B, M, N, K, C, ldc, splits, partial, cv, &g);
+    if (st != PF_OK) return st;
+    const GemmParams& p = g.p;
+    cudaError_t e = g.bn == 64    ? launch_gemm<64>(g.ta, g.tb, p, g.grid, stream)
+                    : g.bn == 128 ? launch_gemm<128>(g.ta, g.tb, p, g.grid, stream)
+                                  : launch_gemm<256>(g.ta, g.tb, p, g.grid, stream);
     if (e != cudaSuccess) return PF_ERR_CUDA;
     if (deferred_splits) {           // the caller sums the slices (together with another product's)
         *deferred_splits = p.splits;
@@ -349,6 +392,41 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
         e = splitk_reduce(partial, C, ldc, M, N, p.splits, PF_BF16, stream);
         if (e != cudaSuccess) return PF_ERR_CUDA;
     }
+    return PF_OK;
+}
+
+template <int BN>
+cudaError_t launch_gemm2(const GemmLaunch& a, const GemmLaunch& b, cudaStream_t stream) {
+    constexpr size_t smem = 1024 + 1024 + static_cast<size_t>(kStages) * (kBM * kBK * 2 + BN * kBK * 2);
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    const int ca = static_cast<int>(a.grid.x * a.grid.y * a.grid.z), cb = static_cast<int>(b.grid.x * b.grid.y * b.grid.z);
+    const int2 ta = make_int2(a.grid.x, a.grid.y), tb = make_int2(b.grid.x, b.grid.y);
+    cudaError_t e = launch_overlapped(tc_gemm2_kernel<BN>, dim3(ca + cb), dim3(kGemmThreads), smem, stream, a.ta, a.tb,
+                                      b.ta, b.tb, a.p, b.p, ca, ta, tb);
+    if (e == cudaSuccess) count_launch();
+    return e;
+}
+
+// Both factor gradients of a layer in one launch, then one launch that sums their slices.
+int gemm_pair_split(const GemmLaunch& a, void* Ca, int64_t ldca, float* pa, const GemmLaunch& b, void* Cb, int64_t ldcb,
+                    float* pb, cudaStream_t stream) {
+    if (a.bn != b.bn || a.bn == 256) return PF_ERR_UNSUPPORTED;
+    const cudaError_t e = a.bn == 64 ? launch_gemm2<64>(a, b, stream) : launch_gemm2<128>(a, b, stream);
+    if (e != cudaSuccess) return PF_ERR_CUDA;
+    const int su = a.p.splits, sv = b.p.splits;
+    if (su > 1 && sv > 1)
+        return splitk_reduce2_bf16(pa, Ca, ldca, a.p.M, a.p.N, su, pb, Cb, ldcb, b.p.M, b.p.N, sv, stream) == cudaSuccess
+                   ? PF_OK : PF_ERR_CUDA;
+    if (su > 1 && splitk_reduce(pa, Ca, ldca, a.p.M, a.p.N, su, PF_BF16, stream) != cudaSuccess) return PF_ERR_CUDA;
+    if (sv > 1 && splitk_reduce(pb, Cb, ldcb, b.p.M, b.p.N, sv, PF_BF16, stream) != cudaSuccess) return PF_ERR_CUDA;
     return PF_OK;
 }
 
@@ -492,6 +570,13 @@ int linear_bwd(const LinearArgs& a, int* handled) {
             if (st != PF_OK) return st;
         }
     }
+    {   // dU = x^T G and dV = dY^T T: one launch for both products, one for their slice sums
+        GemmLaunch gu, gv;
+        if (gemm_prepare({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, nullptr, &gu) == PF_OK &&
+            gemm_prepare({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, nullptr, &gv) == PF_OK &&
+            gu.bn == gv.bn && gu.bn != 256)
+            return gemm_pair_split(gu, a.dU, a.lddu, pu, gv, a.dV, a.lddv, pv, a.stream);
+    }
     if (su > 1 && sv > 1) {
         // both factor gradients are split over m: one launch sums the slices of both
         int used_u = 0, used_v = 0;
@@ -580,20 +665,13 @@ int conv_bwd(const ConvArgs& a, int* handled) {
         if (st != PF_OK) return st;
     }
     // dU[tap] = shifted x^T dT ; dV = dY^T T   (reductions over all pixels, split across CTAs)
-    int used_u = 0, used_v = 0;
     const ConvA cu{2, a.N, a.H, a.W, a.C, a.kw, a.pad, a.C};
-    st = gemm({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, a.stream, &used_u, &cu);
+    GemmLaunch gu, gv;
+    st = gemm_prepare({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, &cu, &gu);
     if (st != PF_OK) return st;
-    st = gemm({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, a.stream, &used_v);
+    st = gemm_prepare({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, nullptr, &gv);
     if (st != PF_OK) return st;
-    if (used_u > 1 && used_v > 1)
-        return splitk_reduce2_bf16(pu, a.dU, a.R, Keff, a.R, used_u, pv, a.dV, a.R, a.O, a.R, used_v, a.stream) ==
-                       cudaSuccess ? PF_OK : PF_ERR_CUDA;
-    if (used_u > 1 && splitk_reduce(pu, a.dU, a.R, Keff, a.R, used_u, PF_BF16, a.stream) != cudaSuccess)
-        return PF_ERR_CUDA;
-    if (used_v > 1 && splitk_reduce(pv, a.dV, a.R, a.O, a.R, used_v, PF_BF16, a.stream) != cudaSuccess)
-        return PF_ERR_CUDA;
-    return PF_OK;
+    return gemm_pair_split(gu, a.dU, a.R, pu, gv, a.dV, a.R, pv, a.stream);
 }
 
 }  // namespace tc
