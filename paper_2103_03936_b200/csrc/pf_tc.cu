@@ -313,6 +313,26 @@ int pick_splits(int64_t M, int64_t N, int bn, int64_t K) {
 }
 int pick_bn(int64_t N) { return N <= 64 ? 64 : 128; }
 
+// Slice counts for two products that share one launch (dU: Mu x N, dV: Mv x N, both contracting
+// over K): all CTAs should fit one wave and finish together, so the longest CTA (in k-blocks) is
+// minimised subject to tiles_u * su + tiles_v * sv <= SM count.
+void pick_pair_splits(int64_t Mu, int64_t Mv, int64_t N, int64_t K, int kblock, int* su, int* sv) {
+    const int bn = pick_bn(N);
+    const int64_t tu = ceil_div(Mu, kBM) * ceil_div(N, bn), tv = ceil_div(Mv, kBM) * ceil_div(N, bn);
+    const int64_t nkb = ceil_div(K, kblock);
+    *su = 1; *sv = 1;
+    if (tu < 1 || tv < 1 || nkb < 1 || tu + tv > kNumSMs) return;
+    int64_t best = nkb + 1;
+    for (int64_t a = 1; a <= 64 && a <= nkb && tu * a + tv <= kNumSMs; ++a) {
+        int64_t b = (kNumSMs - tu * a) / tv;
+        if (b > 64) b = 64;
+        if (b > nkb) b = nkb;
+        if (b < 1) continue;
+        const int64_t longest = std::max(ceil_div(nkb, a), ceil_div(nkb, b));
+        if (longest < best) { best = longest; *su = static_cast<int>(a); *sv = static_cast<int>(b); }
+    }
+}
+
 // C[M,N] (bf16, ldc) = A * B.  `partial` must hold splits*M*N floats when splits > 1.
 struct ConvA {
     int mode;                   // 1: dX (A = dT image), 2: dU (A = x image)
@@ -468,7 +488,8 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
     if (bwd) {
         b += repack_room(m, n);                                             // dY
         b += align_up(static_cast<size_t>(m) * pad8(r) * 2, 256);           // G at padded pitch
-        const int su = pick_splits(k, r, pick_bn(r), m), sv = pick_splits(n, r, pick_bn(r), m);
+        int su, sv;
+        pick_pair_splits(k, n, r, m, kBK, &su, &sv);
         const size_t pu = su > 1 ? static_cast<size_t>(su) * k * r * 4 : 0;
         const size_t pv = sv > 1 ? static_cast<size_t>(sv) * n * r * 4 : 0;
         b += align_up(pu, 256) + align_up(pv, 256);
@@ -545,7 +566,8 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     char* G = scratch;
     const int64_t ldG = pad8(a.r);
     scratch += align_up(static_cast<size_t>(a.m) * ldG * 2, 256);
-    const int su = pick_splits(a.k, a.r, pick_bn(a.r), a.m), sv = pick_splits(a.n, a.r, pick_bn(a.r), a.m);
+    int su, sv;
+    pick_pair_splits(a.k, a.n, a.r, a.m, kBK, &su, &sv);
     float* pu = reinterpret_cast<float*>(scratch);
     scratch += align_up(su > 1 ? static_cast<size_t>(su) * a.k * a.r * 4 : 0, 256);
     float* pv = reinterpret_cast<float*>(scratch);
@@ -614,7 +636,8 @@ size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, in
     if (!bwd) return 0;
     // split partials of dU ((kh*kw*C) x R) and dV (O x R)
     const int64_t P = static_cast<int64_t>(N) * H * W, Keff = static_cast<int64_t>(kh) * kw * C;
-    const int su = pick_splits(Keff, R, pick_bn(R), P), sv = pick_splits(O, R, pick_bn(R), P);
+    int su, sv;
+    pick_pair_splits(Keff, O, R, P, conv_box_h(H, W, 64) * W, &su, &sv);
     (void)stride; (void)pad;
     return align_up(su > 1 ? static_cast<size_t>(su) * Keff * R * 4 : 0, 256) +
            align_up(sv > 1 ? static_cast<size_t>(sv) * O * R * 4 : 0, 256);
@@ -651,7 +674,8 @@ int conv_bwd(const ConvArgs& a, int* handled) {
         T = a.ws_T;
     }
     void* dT = a.ws_G;
-    const int su = pick_splits(Keff, a.R, pick_bn(a.R), M), sv = pick_splits(a.O, a.R, pick_bn(a.R), M);
+    int su, sv;
+    pick_pair_splits(Keff, a.O, a.R, M, conv_box_h(a.H, a.W, 64) * a.W, &su, &sv);
     float* pu = reinterpret_cast<float*>(a.ws);
     float* pv = reinterpret_cast<float*>(a.ws + align_up(su > 1 ? static_cast<size_t>(su) * Keff * a.R * 4 : 0, 256));
     // dT = dY V  (per pixel)
