@@ -143,6 +143,7 @@ int pf_last_device_status(void) {
     if (v != 0) {
         const unsigned int zero = 0;
         if (cudaMemcpy(p, &zero, sizeof(zero), cudaMemcpyHostToDevice) != cudaSuccess) return PF_ERR_CUDA;
+        tc::reset_fix_counters();
     }
     return v == 0 ? PF_OK : PF_ERR_TIMEOUT;
 }

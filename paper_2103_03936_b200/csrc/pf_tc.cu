@@ -13,6 +13,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <atomic>
 
 #include "pf_tc_host.h"
 #include "pf_tc_prims.cuh"
@@ -23,15 +24,22 @@ namespace {
 
 constexpr int kBM = 128;       // rows of the output tile = TMEM lanes
 constexpr int kBK = 64;        // contraction elements per pipeline stage (128 bytes of bf16)
-constexpr int kStages = 4;
+constexpr int kMaxStages = 6;
 constexpr int kGemmThreads = 192;
+constexpr int kFixSlots = 32;  // counter sets handed out round-robin to launches that split a contraction
+constexpr int kFixTiles = 160; // output tiles of one split product (tiles * slices never exceeds the SM count)
+
+// Arrival / departure counters of the in-kernel slice sum, two per output tile.  They are zero
+// between launches: the last CTA to leave a tile clears its pair.
+__device__ unsigned int g_fix_counters[kFixSlots][kFixTiles * 2];
 
 struct GemmCtl {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     uint64_t tmem_full;
     uint32_t tmem_base;
     uint32_t abort;
+    uint32_t fix_ok;
 };
 
 struct GemmParams {
@@ -39,9 +47,12 @@ struct GemmParams {
     int a_mn, b_mn;          // 1 = operand stored with the M/N index contiguous
     int kb_per_split;        // k-blocks handled by one z-slice
     int splits;
-    void* C;                 // bf16 [M, ldc] when splits == 1
+    int num_stages;
+    int tiles_x;             // row tiles of this product (tile id = column tile * tiles_x + row tile)
+    void* C;                 // bf16 [M, ldc]
     long long ldc;
-    float* partial;          // fp32 [splits, M, N] when splits > 1
+    float* partial;          // splits > 1: fp32 slices, one 128 x BN block per (tile, slice)
+    unsigned int* counters;  // splits > 1: two counters per tile
     unsigned int* status;
     // Implicit-GEMM convolution operand A (tmA is then a 4-D NHWC map):
     //   conv_mode 1 (dX): A K-major; row tile = cv_box_h full-width image rows of dT; k-block =
@@ -54,39 +65,20 @@ struct GemmParams {
     int nkb_total;           // k-blocks of the whole contraction
 };
 
-__device__ __forceinline__ void store_row_chunk_bf16(__nv_bfloat16* dst, const uint32_t (&v)[32], int ncols,
-                                                      bool vec_ok) {
-    if (ncols == 32 && vec_ok) {
-        uint4* d4 = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            uint4 o;
-            o.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1]));
-            o.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3]));
-            o.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5]));
-            o.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]));
-            d4[q] = o;
-        }
-    } else {
-#pragma unroll
-        for (int c = 0; c < 32; ++c)
-            if (c < ncols) dst[c] = __float2bfloat16_rn(__uint_as_float(v[c]));
-    }
-}
-__device__ __forceinline__ void store_row_chunk_f32(float* dst, const uint32_t (&v)[32], int ncols, bool vec_ok) {
-    if (ncols == 32 && vec_ok) {
-        float4* d4 = reinterpret_cast<float4*>(dst);
-#pragma unroll
-        for (int q = 0; q < 8; ++q)
-            d4[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
-                                __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
-    } else {
-#pragma unroll
-        for (int c = 0; c < 32; ++c)
-            if (c < ncols) dst[c] = __uint_as_float(v[c]);
-    }
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
+// One output tile (128 rows x BN columns) of C = A * B, or one slice of its contraction.
+//
+// Epilogue.  Unsplit: each epilogue warp turns its 32 accumulator rows into bf16, transposes them
+// through a padded shared-memory panel and writes whole 128-byte row segments (any pitch, any
+// alignment, clipped at the matrix edge).  Split: the fp32 slice goes to the workspace in the
+// order [32-column chunk][4-column group][row][4], which makes every store instruction of a warp
+// one contiguous 512-byte run; then the CTAs of a tile meet at a counter and each sums, in slice
+// order, its share of the rows over all slices and writes bf16 (bit-reproducible, no second launch).
 template <int BN>
 __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
                                           const int bx, const int by, const int bz) {
@@ -106,14 +98,17 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     const int kb_beg = bz * p.kb_per_split;
     const int kb_end = min(nkb_total, kb_beg + p.kb_per_split);
     const int nkb = kb_end - kb_beg;
+    const uint32_t NS = static_cast<uint32_t>(p.num_stages);
+    const int tile = by * p.tiles_x + bx;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (uint32_t s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->tmem_full), 1);
         ctl->abort = 0;
+        ctl->fix_ok = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
         tma_prefetch_desc(&tmA);
@@ -122,7 +117,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     if (p.conv_mode == 2 && p.kpix < 64) {
         // k-blocks hold fewer than 64 pixels: the unused contraction rows of every A stage must be
         // zero (TMA never writes them), so that they add nothing to the sum
-        for (int i = threadIdx.x; i < kStages * static_cast<int>(kABytes / 16); i += blockDim.x) {
+        for (int i = threadIdx.x; i < static_cast<int>(NS) * static_cast<int>(kABytes / 16); i += blockDim.x) {
             const int st = i / static_cast<int>(kABytes / 16), off = i - st * static_cast<int>(kABytes / 16);
             *reinterpret_cast<uint4*>(tiles + st * kStageBytes + off * 16) = make_uint4(0, 0, 0, 0);
         }
@@ -158,7 +153,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                     const int h0 = (bx - img * p.cv_tpi) * p.cv_box_h;
                     tma_load_4d(a_dst, &tmA, full, rb * 64, p.cv_pad - tb, h0 + p.cv_pad - ta, img);
                     tma_load_2d(b_dst, &tmB, full, rb * 64, tap * p.cv_C + n0);
-                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                    if (++s == NS) { s = 0; ph ^= 1u; }
                     continue;
                 }
                 if (p.conv_mode == 2) {
@@ -171,7 +166,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                     tma_load_4d(a_dst + 8192, &tmA, full, c0 + 64, tb - p.cv_pad, h0 + ta - p.cv_pad, img);
 #pragma unroll
                     for (int h = 0; h < BN / 64; ++h) tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, kbg * p.kpix);
-                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                    if (++s == NS) { s = 0; ph ^= 1u; }
                     continue;
                 } else if (p.a_mn) {
                     tma_load_2d(a_dst, &tmA, full, m0, k0);
@@ -185,7 +180,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                 } else {
                     tma_load_2d(b_dst, &tmB, full, k0, n0);
                 }
-                if (++s == kStages) { s = 0; ph ^= 1u; }
+                if (++s == NS) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
@@ -210,7 +205,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                 tc_mma_bf16(tmem_base, a_desc + 2 * a_step, b_desc + 2 * b_step, idesc, 1u);
                 tc_mma_bf16(tmem_base, a_desc + 3 * a_step, b_desc + 3 * b_step, idesc, 1u);
                 tc_commit(smem_u32(&ctl->empty[s]));   // frees the stage once these MMAs have read it
-                if (++s == kStages) { s = 0; ph ^= 1u; }
+                if (++s == NS) { s = 0; ph ^= 1u; }
             }
             if (ok) tc_commit(smem_u32(&ctl->tmem_full));
         }
@@ -219,28 +214,109 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
         const bool ok = mbar_wait_warp(smem_u32(&ctl->tmem_full), 0, abort_flag, p.status);
         tc_fence_after();
         if (ok) {
-            const int row = m0 + q * 32 + lane;
-            const bool row_ok = row < p.M && q * 32 + lane < p.rows_tile;
-            __nv_bfloat16* crow = nullptr;
-            float* prow = nullptr;
-            bool vec_ok;
+            const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
             if (p.splits > 1) {
-                prow = p.partial + (static_cast<size_t>(bz) * p.M + (row_ok ? row : 0)) * p.N;
-                vec_ok = (p.N % 4) == 0;
-            } else {
-                crow = reinterpret_cast<__nv_bfloat16*>(p.C) + static_cast<size_t>(row_ok ? row : 0) * p.ldc;
-                vec_ok = (p.ldc % 8) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 15) == 0;
-            }
+                float4* blk = reinterpret_cast<float4*>(p.partial) +
+                              (static_cast<size_t>(tile) * p.splits + bz) * (kBM * BN / 4) + (q * 32 + lane);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c * 32, v);
-                tmem_ld_wait();
-                const int col = n0 + c * 32;
-                const int ncols = min(32, p.N - col);
-                if (row_ok && ncols > 0) {
-                    if (p.splits > 1) store_row_chunk_f32(prow + col, v, ncols, vec_ok);
-                    else store_row_chunk_bf16(crow + col, v, ncols, vec_ok);
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(lane_base + c * 32, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        __stcg(blk + (c * 8 + g) * kBM,
+                               make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]),
+                                           __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3])));
+                }
+                __threadfence();
+            } else {
+                // every MMA has completed, so the pipeline stages are free: 32 x 33-word panel per warp
+                uint32_t* stg = reinterpret_cast<uint32_t*>(tiles) + (warp - 2) * (32 * 33);
+                __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
+                const bool pair_ok = (p.ldc % 2) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 3) == 0;
+                const bool vec_ok = (p.ldc % 8) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 15) == 0;
+                if (vec_ok) {
+                    // 16-byte aligned rows: stage 32 rows x 64 columns (128 bytes per row, 16-byte pieces
+                    // XOR-swizzled by the row so that both passes are free of bank conflicts), then
+                    // store four whole 128-byte row segments per instruction
+                    const uint32_t panel = smem_u32(tiles) + static_cast<uint32_t>(warp - 2) * 4096u;
+                    const uint32_t own = panel + static_cast<uint32_t>(lane) * 128u, sw = static_cast<uint32_t>(lane & 7);
+                    const int sub = lane >> 3, piece = lane & 7;
+                    const size_t row_step = static_cast<size_t>(4) * p.ldc;
+#pragma unroll 1
+                    for (int c = 0; c < BN / 64; ++c) {
+                        uint32_t v0[32], v1[32];
+                        tmem_ld32(lane_base + c * 64, v0);
+                        tmem_ld32(lane_base + c * 64 + 32, v1);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(v0[8 * t + 0]), __uint_as_float(v0[8 * t + 1]));
+                            o.y = pack_bf16x2(__uint_as_float(v0[8 * t + 2]), __uint_as_float(v0[8 * t + 3]));
+                            o.z = pack_bf16x2(__uint_as_float(v0[8 * t + 4]), __uint_as_float(v0[8 * t + 5]));
+                            o.w = pack_bf16x2(__uint_as_float(v0[8 * t + 6]), __uint_as_float(v0[8 * t + 7]));
+                            st_shared_v4(own + ((static_cast<uint32_t>(t) ^ sw) << 4), o);
+                            o.x = pack_bf16x2(__uint_as_float(v1[8 * t + 0]), __uint_as_float(v1[8 * t + 1]));
+                            o.y = pack_bf16x2(__uint_as_float(v1[8 * t + 2]), __uint_as_float(v1[8 * t + 3]));
+                            o.z = pack_bf16x2(__uint_as_float(v1[8 * t + 4]), __uint_as_float(v1[8 * t + 5]));
+                            o.w = pack_bf16x2(__uint_as_float(v1[8 * t + 6]), __uint_as_float(v1[8 * t + 7]));
+                            st_shared_v4(own + ((static_cast<uint32_t>(4 + t) ^ sw) << 4), o);
+                        }
+                        __syncwarp();
+                        const int col = n0 + c * 64 + piece * 8;
+                        const int rin0 = q * 32 + sub;
+                        __nv_bfloat16* dst = Cb + static_cast<size_t>(m0 + rin0) * p.ldc + col;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int rr = i * 4 + sub, rin_i = rin0 + i * 4;
+                            const uint4 w = ld_shared_v4(panel + static_cast<uint32_t>(rr) * 128u +
+                                                         ((static_cast<uint32_t>(piece) ^ static_cast<uint32_t>(rr & 7)) << 4));
+                            if (m0 + rin_i < p.M && rin_i < p.rows_tile) {
+                                if (col + 8 <= p.N) {
+                                    *reinterpret_cast<uint4*>(dst) = w;
+                                } else {
+                                    const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e)
+                                        if (col + e < p.N)
+                                            dst[e] = __ushort_as_bfloat16(static_cast<unsigned short>((ws[e >> 1] >> ((e & 1) * 16)) & 0xffffu));
+                                }
+                            }
+                            dst += row_step;
+                        }
+                        __syncwarp();
+                    }
+                } else
+#pragma unroll 1
+                for (int c = 0; c < BN / 64; ++c) {
+                    uint32_t v0[32], v1[32];
+                    tmem_ld32(lane_base + c * 64, v0);
+                    tmem_ld32(lane_base + c * 64 + 32, v1);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int w = 0; w < 16; ++w) {
+                        stg[lane * 33 + w] = pack_bf16x2(__uint_as_float(v0[2 * w]), __uint_as_float(v0[2 * w + 1]));
+                        stg[lane * 33 + 16 + w] = pack_bf16x2(__uint_as_float(v1[2 * w]), __uint_as_float(v1[2 * w + 1]));
+                    }
+                    __syncwarp();
+                    const int col = n0 + c * 64 + 2 * lane;
+#pragma unroll 4
+                    for (int j = 0; j < 32; ++j) {
+                        const int rj = q * 32 + j, rowj = m0 + rj;
+                        if (rowj < p.M && rj < p.rows_tile) {
+                            const uint32_t w = stg[j * 33 + lane];
+                            __nv_bfloat16* dst = Cb + static_cast<size_t>(rowj) * p.ldc + col;
+                            if (pair_ok && col + 1 < p.N) {
+                                *reinterpret_cast<uint32_t*>(dst) = w;
+                            } else {
+                                if (col < p.N) dst[0] = __ushort_as_bfloat16(static_cast<unsigned short>(w & 0xffffu));
+                                if (col + 1 < p.N) dst[1] = __ushort_as_bfloat16(static_cast<unsigned short>(w >> 16));
+                            }
+                        }
+                    }
+                    __syncwarp();
                 }
             }
         }
@@ -248,10 +324,90 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, BN);
+    if (p.splits <= 1) return;
+
+    // ---- slice sum: wait until every slice of this tile is in the workspace, then sum a share of rows
+    unsigned int* cnt = p.counters + 2 * tile;
+    if (threadIdx.x == 0) {
+        uint32_t good = (*abort_flag == 0u) ? 1u : 0u;
+        if (good) {
+            __threadfence();
+            const unsigned int before = atomicAdd(cnt, 1u);
+            const long long t0 = clock64();
+            while (before + 1u < static_cast<unsigned int>(p.splits) &&
+                   ld_acquire_gpu(cnt) < static_cast<unsigned int>(p.splits)) {
+                if (clock64() - t0 > kWaitCycleLimit) {
+                    good = 0u;
+                    if (p.status) atomicExch(p.status, kStatusTimeout);
+                    break;
+                }
+            }
+            __threadfence();
+        }
+        ctl->fix_ok = good;
+    }
+    __syncthreads();
+    if (ctl->fix_ok) {
+        const int S = p.splits;
+        const int rows_per = (kBM + S - 1) / S;
+        const int r_beg = bz * rows_per;
+        const int nrows = min(kBM, r_beg + rows_per) - r_beg;
+        const float4* base = reinterpret_cast<const float4*>(p.partial) + static_cast<size_t>(tile) * S * (kBM * BN / 4);
+        __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
+        // Two items (row, 4-column group) per thread and pass, eight slices of each in flight at a
+        // time: the sum is bound by L2 latency, so the loads are issued before any of them is used.
+        const int items = nrows * (BN / 4);
+        for (int id0 = threadIdx.x; id0 < items; id0 += 2 * kGemmThreads) {
+            const int id1 = id0 + kGemmThreads;
+            const bool two = id1 < items;
+            const int g0 = id0 / nrows, rr0 = r_beg + (id0 - g0 * nrows);
+            const int g1 = two ? id1 / nrows : g0, rr1 = two ? r_beg + (id1 - g1 * nrows) : rr0;
+            const float4* src0 = base + g0 * kBM + rr0;
+            const float4* src1 = base + g1 * kBM + rr1;
+            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+            for (int s0 = 0; s0 < S; s0 += 8) {
+                float4 t0[8], t1[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int s = min(s0 + u, S - 1);
+                    t0[u] = __ldcg(src0 + static_cast<size_t>(s) * (kBM * BN / 4));
+                    t1[u] = __ldcg(src1 + static_cast<size_t>(s) * (kBM * BN / 4));
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (s0 + u < S) {
+                        a0.x += t0[u].x; a0.y += t0[u].y; a0.z += t0[u].z; a0.w += t0[u].w;
+                        a1.x += t1[u].x; a1.y += t1[u].y; a1.z += t1[u].z; a1.w += t1[u].w;
+                    }
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                if (h == 1 && !two) break;
+                const float4 acc = h ? a1 : a0;
+                const int row = m0 + (h ? rr1 : rr0), col = n0 + (h ? g1 : g0) * 4;
+                if (row < p.M) {
+                    __nv_bfloat16* dst = Cb + static_cast<size_t>(row) * p.ldc + col;
+                    if (col < p.N) dst[0] = __float2bfloat16_rn(acc.x);
+                    if (col + 1 < p.N) dst[1] = __float2bfloat16_rn(acc.y);
+                    if (col + 2 < p.N) dst[2] = __float2bfloat16_rn(acc.z);
+                    if (col + 3 < p.N) dst[3] = __float2bfloat16_rn(acc.w);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && ctl->fix_ok) {
+        const unsigned int left = atomicAdd(cnt + 1, 1u);
+        if (left + 1u == static_cast<unsigned int>(p.splits)) {   // every slice has read what it needs
+            cnt[0] = 0u;
+            cnt[1] = 0u;
+            __threadfence();
+        }
+    }
 }
 
 template <int BN>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kGemmThreads, BN <= 128 ? 2 : 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const GemmParams p) {
     gemm_tile<BN>(tmA, tmB, p, blockIdx.x, blockIdx.y, blockIdx.z);
@@ -262,7 +418,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // from its linear index.  One launch pays the start-up latency once and packs the short CTAs of
 // one problem into the tail of the other.
 template <int BN>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kGemmThreads, BN <= 128 ? 2 : 1)
 tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                 const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
                 const GemmParams p0, const GemmParams p1, const int ctas_a, const int2 tiles_a, const int2 tiles_b) {
@@ -283,22 +439,59 @@ struct Operand {
     bool mn_major;
 };
 
+size_t gemm_smem(int bn, int stages) {
+    return 1024 + 1024 + static_cast<size_t>(stages) * (kBM * kBK * 2 + bn * kBK * 2);
+}
+// Pipeline depth: a grid that fits one wave gets every stage shared memory has room for; a
+// larger grid gets stages small enough for two CTAs per SM, so that the prologue and epilogue of
+// one CTA overlap the main loop of the other.
+int pick_stages(int bn, int64_t ctas) {
+    const size_t stage = static_cast<size_t>(kBM * kBK * 2 + bn * kBK * 2);
+    const size_t room = (ctas > kNumSMs && bn <= 128) ? (113 * 1024 - 2048) : (200 * 1024 - 2048);
+    int ns = static_cast<int>(room / stage);
+    if (ns > kMaxStages) ns = kMaxStages;
+    if (ns < 2) ns = 2;
+    return ns;
+}
+
 template <int BN>
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, dim3 grid,
                         cudaStream_t stream) {
-    constexpr size_t smem = 1024 + 1024 + static_cast<size_t>(kStages) * (kBM * kBK * 2 + BN * kBK * 2);
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem));
+                                             static_cast<int>(std::min(gemm_smem(BN, kMaxStages), static_cast<size_t>(227 * 1024))));
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    cudaError_t e = launch_overlapped(tc_gemm_kernel<BN>, grid, dim3(kGemmThreads), smem, stream, ta, tb, p);
+    cudaError_t e = launch_overlapped(tc_gemm_kernel<BN>, grid, dim3(kGemmThreads), gemm_smem(BN, p.num_stages), stream,
+                                      ta, tb, p);
     if (e == cudaSuccess) count_launch();
     return e;
+}
+
+// Device address of the counter set a launch may use (sets rotate, so that launches in flight on
+// different streams do not share counters unless more than kFixSlots of them overlap).
+unsigned int* next_fix_counters() {
+    static unsigned int* base[64] = {};
+    static std::atomic<unsigned int> next{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!base[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_fix_counters) != cudaSuccess) return nullptr;
+        base[dev] = static_cast<unsigned int*>(ptr);
+    }
+    return base[dev] + static_cast<size_t>(next.fetch_add(1) % kFixSlots) * (kFixTiles * 2);
+}
+
+// Workspace floats of a split product: one 128 x bn block per (tile, slice).
+size_t partial_bytes(int64_t M, int64_t N, int splits) {
+    if (splits <= 1) return 0;
+    const int bn = N <= 64 ? 64 : 128;
+    return static_cast<size_t>(ceil_div(M, kBM) * ceil_div(N, bn)) * splits * kBM * bn * 4;
 }
 
 int pick_splits(int64_t M, int64_t N, int bn, int64_t K) {
@@ -388,66 +581,63 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     dim3 grid(static_cast<unsigned>(ceil_div(M, p.rows_tile)), static_cast<unsigned>(ceil_div(N, bn)),
               static_cast<unsigned>(p.splits));
     if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
+    p.tiles_x = static_cast<int>(grid.x);
+    p.num_stages = pick_stages(bn, static_cast<int64_t>(grid.x) * grid.y * grid.z);
+    p.counters = nullptr;
+    if (p.splits > 1) {
+        // the CTAs of a tile wait for one another, so all of them must be resident at once
+        if (static_cast<int64_t>(grid.x) * grid.y > kFixTiles || static_cast<int64_t>(grid.x) * grid.y * grid.z > kNumSMs ||
+            bn == 256 || partial == nullptr)
+            return PF_ERR_UNSUPPORTED;
+        p.counters = next_fix_counters();
+        if (!p.counters) return PF_ERR_CUDA;
+    }
     out->grid = grid;
     out->bn = bn;
     return PF_OK;
 }
 
 int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
-         int splits, float* partial, cudaStream_t stream, int* deferred_splits = nullptr,
-         const ConvA* cv = nullptr) {
+         int splits, float* partial, cudaStream_t stream, const ConvA* cv = nullptr) {
     GemmLaunch g;
-    const int st = gemm_prepare(A, B, M, N, K, C, ldc, splits, partial, cv, &g);
+    int st = gemm_prepare(A, B, M, N, K, C, ldc, splits, partial, cv, &g);
+    if (st == PF_ERR_UNSUPPORTED && splits > 1) st = gemm_prepare(A, B, M, N, K, C, ldc, 1, nullptr, cv, &g);
     if (st != PF_OK) return st;
     const GemmParams& p = g.p;
     cudaError_t e = g.bn == 64    ? launch_gemm<64>(g.ta, g.tb, p, g.grid, stream)
                     : g.bn == 128 ? launch_gemm<128>(g.ta, g.tb, p, g.grid, stream)
                                   : launch_gemm<256>(g.ta, g.tb, p, g.grid, stream);
-    if (e != cudaSuccess) return PF_ERR_CUDA;
-    if (deferred_splits) {           // the caller sums the slices (together with another product's)
-        *deferred_splits = p.splits;
-        return PF_OK;
-    }
-    if (p.splits > 1) {
-        e = splitk_reduce(partial, C, ldc, M, N, p.splits, PF_BF16, stream);
-        if (e != cudaSuccess) return PF_ERR_CUDA;
-    }
-    return PF_OK;
+    return e == cudaSuccess ? PF_OK : PF_ERR_CUDA;
 }
 
 template <int BN>
 cudaError_t launch_gemm2(const GemmLaunch& a, const GemmLaunch& b, cudaStream_t stream) {
-    constexpr size_t smem = 1024 + 1024 + static_cast<size_t>(kStages) * (kBM * kBK * 2 + BN * kBK * 2);
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem));
+                                             static_cast<int>(std::min(gemm_smem(BN, kMaxStages), static_cast<size_t>(227 * 1024))));
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
     const int ca = static_cast<int>(a.grid.x * a.grid.y * a.grid.z), cb = static_cast<int>(b.grid.x * b.grid.y * b.grid.z);
     const int2 ta = make_int2(a.grid.x, a.grid.y), tb = make_int2(b.grid.x, b.grid.y);
-    cudaError_t e = launch_overlapped(tc_gemm2_kernel<BN>, dim3(ca + cb), dim3(kGemmThreads), smem, stream, a.ta, a.tb,
-                                      b.ta, b.tb, a.p, b.p, ca, ta, tb);
+    // both products run with the pipeline depth of the whole launch
+    GemmParams pa = a.p, pb = b.p;
+    if ((pa.splits > 1 || pb.splits > 1) && ca + cb > kNumSMs) return cudaErrorInvalidConfiguration;
+    pa.num_stages = pb.num_stages = pick_stages(BN, ca + cb);
+    cudaError_t e = launch_overlapped(tc_gemm2_kernel<BN>, dim3(ca + cb), dim3(kGemmThreads), gemm_smem(BN, pa.num_stages),
+                                      stream, a.ta, a.tb, b.ta, b.tb, pa, pb, ca, ta, tb);
     if (e == cudaSuccess) count_launch();
     return e;
 }
 
-// Both factor gradients of a layer in one launch, then one launch that sums their slices.
-int gemm_pair_split(const GemmLaunch& a, void* Ca, int64_t ldca, float* pa, const GemmLaunch& b, void* Cb, int64_t ldcb,
-                    float* pb, cudaStream_t stream) {
+// Both factor gradients of a layer in one launch (their slices are summed inside the kernel).
+int gemm_pair(const GemmLaunch& a, const GemmLaunch& b, cudaStream_t stream) {
     if (a.bn != b.bn || a.bn == 256) return PF_ERR_UNSUPPORTED;
     const cudaError_t e = a.bn == 64 ? launch_gemm2<64>(a, b, stream) : launch_gemm2<128>(a, b, stream);
-    if (e != cudaSuccess) return PF_ERR_CUDA;
-    const int su = a.p.splits, sv = b.p.splits;
-    if (su > 1 && sv > 1)
-        return splitk_reduce2_bf16(pa, Ca, ldca, a.p.M, a.p.N, su, pb, Cb, ldcb, b.p.M, b.p.N, sv, stream) == cudaSuccess
-                   ? PF_OK : PF_ERR_CUDA;
-    if (su > 1 && splitk_reduce(pa, Ca, ldca, a.p.M, a.p.N, su, PF_BF16, stream) != cudaSuccess) return PF_ERR_CUDA;
-    if (sv > 1 && splitk_reduce(pb, Cb, ldcb, b.p.M, b.p.N, sv, PF_BF16, stream) != cudaSuccess) return PF_ERR_CUDA;
-    return PF_OK;
+    return e == cudaSuccess ? PF_OK : PF_ERR_CUDA;
 }
 
 // A row-major bf16 matrix that TMA must read: used as is when 16-byte aligned with a pitch that is
@@ -490,13 +680,11 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
         b += align_up(static_cast<size_t>(m) * pad8(r) * 2, 256);           // G at padded pitch
         int su, sv;
         pick_pair_splits(k, n, r, m, kBK, &su, &sv);
-        const size_t pu = su > 1 ? static_cast<size_t>(su) * k * r * 4 : 0;
-        const size_t pv = sv > 1 ? static_cast<size_t>(sv) * n * r * 4 : 0;
-        b += align_up(pu, 256) + align_up(pv, 256);
+        b += align_up(partial_bytes(k, r, su), 256) + align_up(partial_bytes(n, r, sv), 256);
     }
     // skinny batches: the m x r products (x U, dY V) are split over their contraction to fill the SMs
     const int s1 = std::max(pick_splits(m, r, pick_bn(r), k), bwd ? pick_splits(m, r, pick_bn(r), n) : 1);
-    b += align_up(s1 > 1 ? static_cast<size_t>(s1) * m * r * 4 : 0, 256);
+    b += align_up(partial_bytes(m, r, s1), 256);
     return b;
 }
 
@@ -569,9 +757,9 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     int su, sv;
     pick_pair_splits(a.k, a.n, a.r, a.m, kBK, &su, &sv);
     float* pu = reinterpret_cast<float*>(scratch);
-    scratch += align_up(su > 1 ? static_cast<size_t>(su) * a.k * a.r * 4 : 0, 256);
+    scratch += align_up(partial_bytes(a.k, a.r, su), 256);
     float* pv = reinterpret_cast<float*>(scratch);
-    scratch += align_up(sv > 1 ? static_cast<size_t>(sv) * a.n * a.r * 4 : 0, 256);
+    scratch += align_up(partial_bytes(a.n, a.r, sv), 256);
     float* p1 = reinterpret_cast<float*>(scratch);
     // G = dY V ; dX = G U^T ; dU = x^T G ; dV = dY^T T
     if (need_T) {   // no stash: recompute T = x U
@@ -592,32 +780,22 @@ int linear_bwd(const LinearArgs& a, int* handled) {
             if (st != PF_OK) return st;
         }
     }
-    {   // dU = x^T G and dV = dY^T T: one launch for both products, one for their slice sums
+    {   // dU = x^T G and dV = dY^T T: one launch for both products when their tiles match
         GemmLaunch gu, gv;
         if (gemm_prepare({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, nullptr, &gu) == PF_OK &&
             gemm_prepare({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, nullptr, &gv) == PF_OK &&
             gu.bn == gv.bn && gu.bn != 256)
-            return gemm_pair_split(gu, a.dU, a.lddu, pu, gv, a.dV, a.lddv, pv, a.stream);
-    }
-    if (su > 1 && sv > 1) {
-        // both factor gradients are split over m: one launch sums the slices of both
-        int used_u = 0, used_v = 0;
-        st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream, &used_u);
-        if (st != PF_OK) return st;
-        st = gemm({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, a.stream, &used_v);
-        if (st != PF_OK) return st;
-        if (used_u > 1 && used_v > 1)
-            return splitk_reduce2_bf16(pu, a.dU, a.lddu, a.k, a.r, used_u, pv, a.dV, a.lddv, a.n, a.r, used_v,
-                                       a.stream) == cudaSuccess ? PF_OK : PF_ERR_CUDA;
-        if (used_u > 1 && splitk_reduce(pu, a.dU, a.lddu, a.k, a.r, used_u, PF_BF16, a.stream) != cudaSuccess)
-            return PF_ERR_CUDA;
-        if (used_v > 1 && splitk_reduce(pv, a.dV, a.lddv, a.n, a.r, used_v, PF_BF16, a.stream) != cudaSuccess)
-            return PF_ERR_CUDA;
-        return PF_OK;
+            return gemm_pair(gu, gv, a.stream);
     }
     st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream);
     if (st != PF_OK) return st;
     return gemm({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, a.stream);
+}
+
+// After a bounded wait has expired some CTAs may have left their tile counters non-zero.
+void reset_fix_counters() {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_fix_counters) == cudaSuccess) cudaMemset(ptr, 0, sizeof(unsigned int) * kFixSlots * kFixTiles * 2);
 }
 
 // Tensor-core envelope of the factorized convolution: stride 1, "same" padding, channel counts
@@ -639,8 +817,7 @@ size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, in
     int su, sv;
     pick_pair_splits(Keff, O, R, P, conv_box_h(H, W, 64) * W, &su, &sv);
     (void)stride; (void)pad;
-    return align_up(su > 1 ? static_cast<size_t>(su) * Keff * R * 4 : 0, 256) +
-           align_up(sv > 1 ? static_cast<size_t>(sv) * O * R * 4 : 0, 256);
+    return align_up(partial_bytes(Keff, R, su), 256) + align_up(partial_bytes(O, R, sv), 256);
 }
 
 int conv_fwd(const ConvArgs& a, int* handled) {
@@ -677,7 +854,7 @@ int conv_bwd(const ConvArgs& a, int* handled) {
     int su, sv;
     pick_pair_splits(Keff, a.O, a.R, M, conv_box_h(a.H, a.W, 64) * a.W, &su, &sv);
     float* pu = reinterpret_cast<float*>(a.ws);
-    float* pv = reinterpret_cast<float*>(a.ws + align_up(su > 1 ? static_cast<size_t>(su) * Keff * a.R * 4 : 0, 256));
+    float* pv = reinterpret_cast<float*>(a.ws + align_up(partial_bytes(Keff, a.R, su), 256));
     // dT = dY V  (per pixel)
     st = gemm({a.dY, a.O, false}, {a.V, a.R, true}, M, a.R, a.O, dT, a.R, 1, nullptr, a.stream);
     if (st != PF_OK) return st;
@@ -685,7 +862,7 @@ int conv_bwd(const ConvArgs& a, int* handled) {
     if (a.dX) {
         const ConvA cx{1, a.N, a.H, a.W, a.R, a.kw, a.pad, a.C};
         st = gemm({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
-                  nullptr, a.stream, nullptr, &cx);
+                  nullptr, a.stream, &cx);
         if (st != PF_OK) return st;
     }
     // dU[tap] = shifted x^T dT ; dV = dY^T T   (reductions over all pixels, split across CTAs)
@@ -695,7 +872,7 @@ int conv_bwd(const ConvArgs& a, int* handled) {
     if (st != PF_OK) return st;
     st = gemm_prepare({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, nullptr, &gv);
     if (st != PF_OK) return st;
-    return gemm_pair_split(gu, a.dU, a.R, pu, gv, a.dV, a.R, pv, a.stream);
+    return gemm_pair(gu, gv, a.stream);
 }
 
 }  // namespace tc

@@ -48,6 +48,7 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
 size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool bwd);
 size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
                             int pad, bool bwd);
+void reset_fix_counters();  // clears the slice-sum counters (after PF_ERR_TIMEOUT)
 int linear_fwd(const LinearArgs& a, int* handled);
 int linear_bwd(const LinearArgs& a, int* handled);
 int conv_fwd(const ConvArgs& a, int* handled);
