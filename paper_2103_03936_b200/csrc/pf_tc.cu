@@ -37,6 +37,7 @@ struct GemmCtl {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
     uint64_t tmem_full;
+    uint64_t fix_full;       // the slices this CTA sums have been copied into shared memory
     uint32_t tmem_base;
     uint32_t abort;
     uint32_t fix_ok;
@@ -107,6 +108,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->tmem_full), 1);
+        mbar_init(smem_u32(&ctl->fix_full), 1);
         ctl->abort = 0;
         ctl->fix_ok = 0;
         fence_barrier_init();
@@ -229,6 +231,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                                make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]),
                                            __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3])));
                 }
+                fence_proxy_async_all();   // the slices are read back by bulk copies (async proxy)
                 __threadfence();
             } else {
                 // every MMA has completed, so the pipeline stages are free: 32 x 33-word panel per warp
@@ -326,16 +329,23 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     if (warp == 1) tmem_dealloc(tmem_base, BN);
     if (p.splits <= 1) return;
 
-    // ---- slice sum: wait until every slice of this tile is in the workspace, then sum a share of rows
+    // ---- slice sum: wait until every slice of this tile is in the workspace, then sum a share of it.
+    // A share is a run of 4-column groups (all 128 rows), contiguous in every slice, so one bulk copy
+    // per slice brings it into the idle pipeline stages: a single trip to L2 for the whole sum.
     unsigned int* cnt = p.counters + 2 * tile;
+    const int S = p.splits;
+    constexpr int kGroups = BN / 4;
+    const int gper = (kGroups + S - 1) / S;
+    const int g_beg = bz * gper;
+    const int ng = max(0, min(kGroups, g_beg + gper) - g_beg);
+    const uint32_t share = static_cast<uint32_t>(ng) * (kBM * 16u);
     if (threadIdx.x == 0) {
         uint32_t good = (*abort_flag == 0u) ? 1u : 0u;
         if (good) {
             __threadfence();
             const unsigned int before = atomicAdd(cnt, 1u);
             const long long t0 = clock64();
-            while (before + 1u < static_cast<unsigned int>(p.splits) &&
-                   ld_acquire_gpu(cnt) < static_cast<unsigned int>(p.splits)) {
+            while (before + 1u < static_cast<unsigned int>(S) && ld_acquire_gpu(cnt) < static_cast<unsigned int>(S)) {
                 if (clock64() - t0 > kWaitCycleLimit) {
                     good = 0u;
                     if (p.status) atomicExch(p.status, kStatusTimeout);
@@ -343,62 +353,55 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                 }
             }
             __threadfence();
+            fence_proxy_async_all();
+            if (good && ng > 0) {
+                const uint32_t bar = smem_u32(&ctl->fix_full);
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(p.partial) +
+                                     (static_cast<size_t>(tile) * S) * (kBM * BN * 4) + static_cast<size_t>(g_beg) * (kBM * 16);
+                mbar_expect_tx(bar, share * static_cast<uint32_t>(S));
+                for (int s = 0; s < S; ++s)
+                    bulk_load(smem_u32(tiles) + static_cast<uint32_t>(s) * share, src + static_cast<size_t>(s) * (kBM * BN * 4),
+                              share, bar);
+                good = mbar_wait(bar, 0, abort_flag, p.status) ? 1u : 0u;
+            }
         }
         ctl->fix_ok = good;
     }
     __syncthreads();
     if (ctl->fix_ok) {
-        const int S = p.splits;
-        const int rows_per = (kBM + S - 1) / S;
-        const int r_beg = bz * rows_per;
-        const int nrows = min(kBM, r_beg + rows_per) - r_beg;
-        const float4* base = reinterpret_cast<const float4*>(p.partial) + static_cast<size_t>(tile) * S * (kBM * BN / 4);
         __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
-        // Two items (row, 4-column group) per thread and pass, eight slices of each in flight at a
-        // time: the sum is bound by L2 latency, so the loads are issued before any of them is used.
-        const int items = nrows * (BN / 4);
-        for (int id0 = threadIdx.x; id0 < items; id0 += 2 * kGemmThreads) {
-            const int id1 = id0 + kGemmThreads;
-            const bool two = id1 < items;
-            const int g0 = id0 / nrows, rr0 = r_beg + (id0 - g0 * nrows);
-            const int g1 = two ? id1 / nrows : g0, rr1 = two ? r_beg + (id1 - g1 * nrows) : rr0;
-            const float4* src0 = base + g0 * kBM + rr0;
-            const float4* src1 = base + g1 * kBM + rr1;
-            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
-            for (int s0 = 0; s0 < S; s0 += 8) {
-                float4 t0[8], t1[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int s = min(s0 + u, S - 1);
-                    t0[u] = __ldcg(src0 + static_cast<size_t>(s) * (kBM * BN / 4));
-                    t1[u] = __ldcg(src1 + static_cast<size_t>(s) * (kBM * BN / 4));
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (s0 + u < S) {
-                        a0.x += t0[u].x; a0.y += t0[u].y; a0.z += t0[u].z; a0.w += t0[u].w;
-                        a1.x += t1[u].x; a1.y += t1[u].y; a1.z += t1[u].z; a1.w += t1[u].w;
-                    }
+        const float4* sm4 = reinterpret_cast<const float4*>(tiles);
+        const uint32_t share4 = share / 16u;
+        // consecutive threads take consecutive rows of one column group: conflict-free 16-byte reads of
+        // shared memory (the other order costs a 5-way bank conflict on every read); each result
+        // leaves as one 8-byte store
+        const bool vec8 = (p.ldc % 4) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 7) == 0;
+        for (int id = threadIdx.x; id < ng * kBM; id += kGemmThreads) {
+            const int gl = id / kBM, rr = id % kBM;
+            float4 acc = sm4[id];
+#pragma unroll 8
+            for (int s = 1; s < S; ++s) {
+                const float4 t = sm4[static_cast<uint32_t>(s) * share4 + static_cast<uint32_t>(id)];
+                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
             }
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                if (h == 1 && !two) break;
-                const float4 acc = h ? a1 : a0;
-                const int row = m0 + (h ? rr1 : rr0), col = n0 + (h ? g1 : g0) * 4;
-                if (row < p.M) {
-                    __nv_bfloat16* dst = Cb + static_cast<size_t>(row) * p.ldc + col;
-                    if (col < p.N) dst[0] = __float2bfloat16_rn(acc.x);
-                    if (col + 1 < p.N) dst[1] = __float2bfloat16_rn(acc.y);
-                    if (col + 2 < p.N) dst[2] = __float2bfloat16_rn(acc.z);
-                    if (col + 3 < p.N) dst[3] = __float2bfloat16_rn(acc.w);
+            const int row = m0 + rr, col = n0 + (g_beg + gl) * 4;
+            if (row < p.M) {
+                __nv_bfloat16* dst = Cb + static_cast<size_t>(row) * p.ldc + col;
+                if (vec8 && col + 3 < p.N) {
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
+                    continue;
                 }
+                if (col < p.N) dst[0] = __float2bfloat16_rn(acc.x);
+                if (col + 1 < p.N) dst[1] = __float2bfloat16_rn(acc.y);
+                if (col + 2 < p.N) dst[2] = __float2bfloat16_rn(acc.z);
+                if (col + 3 < p.N) dst[3] = __float2bfloat16_rn(acc.w);
             }
         }
     }
     __syncthreads();
     if (threadIdx.x == 0 && ctl->fix_ok) {
         const unsigned int left = atomicAdd(cnt + 1, 1u);
-        if (left + 1u == static_cast<unsigned int>(p.splits)) {   // every slice has read what it needs
+        if (left + 1u == static_cast<unsigned int>(S)) {   // every slice has read what it needs
             cnt[0] = 0u;
             cnt[1] = 0u;
             __threadfence();
@@ -588,6 +591,10 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
         // the CTAs of a tile wait for one another, so all of them must be resident at once
         if (static_cast<int64_t>(grid.x) * grid.y > kFixTiles || static_cast<int64_t>(grid.x) * grid.y * grid.z > kNumSMs ||
             bn == 256 || partial == nullptr)
+            return PF_ERR_UNSUPPORTED;
+        // the slices of a CTA's share are gathered in the pipeline stages
+        const int64_t gper = ceil_div(bn / 4, p.splits);
+        if (gper * p.splits * (kBM * 16) > static_cast<int64_t>(p.num_stages) * (kBM * kBK * 2 + bn * kBK * 2))
             return PF_ERR_UNSUPPORTED;
         p.counters = next_fix_counters();
         if (!p.counters) return PF_ERR_CUDA;

@@ -3,7 +3,8 @@
 Used by ``bench.py --suite FILE``: every benchmark configuration (tiny fp32, Transformer FFN,
 LSTM gates in the tight and in a 16-byte-pitch layout, ResNet-style convolutions with the gradient
 pack, and the rank sweep) is timed with CUDA events on rotating buffer sets larger than L2, and
-written as one JSON object per line.  Only timing lives here; parity is the tests' job.
+written as one JSON object per line (fwd_us and bwd_us are each call timed alone, fwd_bwd_us is
+the pair launched back to back).  Only timing lives here; parity is the tests' job.
 """
 from __future__ import annotations
 
@@ -31,26 +32,34 @@ def _rand(shape, dtype, scale=1.0, relu=False, ld=None):
     return buf[:, :cols]
 
 
-def _time(calls_per_set, iters, warmup=3):
-    """calls_per_set: list (one per buffer set) of (fwd_call, bwd_call[, extra_call])."""
+def _time(calls_per_set, iters, warmup=3, repeats=5):
+    """calls_per_set: list (one per buffer set) of (fwd_call, bwd_call[, extra_call]).
+
+    Every call, and the fwd+bwd pair, is timed on its own as `iters` back-to-back launches that
+    rotate through the buffer sets, between two CUDA events (no event between launches, so that
+    consecutive kernels overlap the way they do in a training step); median and minimum over
+    `repeats` such batches.  The last entry of the result is the fwd+bwd pair."""
     ns = len(calls_per_set)
+    ncalls = len(calls_per_set[0])
     for i in range(warmup):
         for c in calls_per_set[i % ns]:
             c()
     torch.cuda.synchronize()
-    evs = []
-    for i in range(iters):
-        cs = calls_per_set[i % ns]
-        e = [torch.cuda.Event(enable_timing=True) for _ in range(len(cs) + 1)]
-        e[0].record()
-        for j, c in enumerate(cs):
-            c()
-            e[j + 1].record()
-        evs.append(e)
-    torch.cuda.synchronize()
+    groups = [(j,) for j in range(ncalls)] + ([(0, 1)] if ncalls >= 2 else [])
     out = []
-    for j in range(len(calls_per_set[0])):
-        ts = sorted(e[j].elapsed_time(e[j + 1]) * 1e3 for e in evs)
+    for grp in groups:
+        ts = []
+        for _ in range(repeats):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(iters):
+                cs = calls_per_set[i % ns]
+                for j in grp:
+                    cs[j]()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3 / iters)
+        ts.sort()
         out.append({"median_us": ts[len(ts) // 2], "min_us": ts[0]})
     return out
 
@@ -61,7 +70,7 @@ def _floors(flops_fwd, bytes_fwd, bytes_bwd, pk):
     return f, b
 
 
-def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=30):
+def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32):
     tdt = torch.bfloat16 if dtype == wl.BF16 else torch.float32
     s = 2 if dtype == wl.BF16 else 4
     code = pf.PF_BF16 if dtype == wl.BF16 else pf.PF_F32
@@ -94,7 +103,7 @@ def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=30):
     bytes_fwd = s * (m * k + m * n + r * (k + n))
     bytes_bwd = s * (m * n + 2 * m * k + 2 * r * (k + n))
     ff, fb = _floors(flops_fwd, bytes_fwd, bytes_bwd, pk)
-    tot = t[0]["median_us"] + t[1]["median_us"]
+    tot = t[-1]["median_us"]
     return {"config": name, "kind": "linear", "m": m, "k": k, "n": n, "r": r, "dtype": dtype,
             "pitch": "padded to 16 B" if pad_pitch else "tight", "buffer_sets": nsets, "launches_fwd_bwd": launches,
             "fwd_us": t[0]["median_us"], "bwd_us": t[1]["median_us"], "fwd_bwd_us": tot,
@@ -137,7 +146,7 @@ def conv_config(name, c, pk, iters=20):
     bytes_fwd = 2 * (M * c.C + M * c.O + c.R * (Keff + c.O))
     bytes_bwd = 2 * (M * c.O + 2 * M * c.C + 2 * c.R * (Keff + c.O))
     ff, fb = _floors(flops_fwd, bytes_fwd, bytes_bwd, pk)
-    tot = t[0]["median_us"] + t[1]["median_us"]
+    tot = t[-1]["median_us"]
     return {"config": name, "kind": "conv", "N": c.N, "H": c.H, "W": c.W, "C": c.C, "R": c.R, "O": c.O,
             "dtype": "bf16", "buffer_sets": nsets, "launches_fwd_bwd_pack": launches,
             "fwd_us": t[0]["median_us"], "bwd_us": t[1]["median_us"], "pack_us": t[2]["median_us"],
@@ -191,7 +200,7 @@ def run(path, pk, only=None):
             emit(conv_config(f"{name} conv", c, pk))
     for r in wl.SWEEP_RANKS:
         if want(f"C5 sweep r={r}"):
-            emit(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=12))
+            emit(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=8))
     # ResNet-18-sized and Transformer-sized factor-gradient lists (Table 4 / Table 3 parameter counts)
     if want("pack ~3.3M elements"):
         emit(pack_config("pack ~3.3M elements", [147457, 16384, 589821, 65536, 1179653, 131072, 1179648, 131071], pk))
