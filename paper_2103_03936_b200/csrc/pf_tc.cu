@@ -49,6 +49,7 @@ struct GemmParams {
     int kb_per_split;        // k-blocks handled by one z-slice
     int splits;
     int num_stages;
+    int bn;                  // columns of an output tile (the kernel's template value; 64 or 128 in a shared launch)
     int tiles_x;             // row tiles of this product (tile id = column tile * tiles_x + row tile)
     void* C;                 // bf16 [M, ldc]
     long long ldc;
@@ -416,21 +417,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     gemm_tile<BN>(tmA, tmB, p, blockIdx.x, blockIdx.y, blockIdx.z);
 }
 
-// Two independent products in one launch (dU = x^T G and dV = dY^T T of one layer): CTAs
-// [0, ctas_a) work on problem a, the rest on problem b; each decodes (row tile, column tile, slice)
-// from its linear index.  One launch pays the start-up latency once and packs the short CTAs of
-// one problem into the tail of the other.
-template <int BN>
-__global__ void __launch_bounds__(kGemmThreads, BN <= 128 ? 2 : 1)
-tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
-                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
-                const GemmParams p0, const GemmParams p1, const int ctas_a, const int2 tiles_a, const int2 tiles_b) {
-    const bool first = static_cast<int>(blockIdx.x) < ctas_a;
-    const int idx = first ? blockIdx.x : blockIdx.x - ctas_a;
-    const int2 t = first ? tiles_a : tiles_b;             // (row tiles, column tiles)
+// Up to three independent products in one launch (dU = x^T G, dV = dY^T T and, where it is a plain
+// product, dX of one layer): CTAs [0, end0) work on product 0, [end0, end1) on product 1, the rest on
+// product 2; each decodes (row tile, column tile, slice) from its linear index.  One launch pays the
+// start-up latency once and packs the short CTAs of one product beside the long ones of another.
+// Tiles may be 64 or 128 columns wide per product.
+__device__ __forceinline__ void gemm_any(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int idx,
+                                         const int2 t) {
     const int bx = idx % t.x, by = (idx / t.x) % t.y, bz = idx / (t.x * t.y);
-    if (first) gemm_tile<BN>(tmA0, tmB0, p0, bx, by, bz);
-    else gemm_tile<BN>(tmA1, tmB1, p1, bx, by, bz);
+    if (p.bn == 64) gemm_tile<64>(tmA, tmB, p, bx, by, bz);
+    else gemm_tile<128>(tmA, tmB, p, bx, by, bz);
+}
+__global__ void __launch_bounds__(kGemmThreads, 2)
+tc_gemm3_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
+                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
+                const GemmParams p0, const GemmParams p1, const GemmParams p2, const int end0, const int end1,
+                const int2 tiles0, const int2 tiles1, const int2 tiles2) {
+    const int idx = blockIdx.x;
+    if (idx < end0) gemm_any(tmA0, tmB0, p0, idx, tiles0);
+    else if (idx < end1) gemm_any(tmA1, tmB1, p1, idx - end0, tiles1);
+    else gemm_any(tmA2, tmB2, p2, idx - end1, tiles2);
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -585,6 +592,7 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
               static_cast<unsigned>(p.splits));
     if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
     p.tiles_x = static_cast<int>(grid.x);
+    p.bn = bn;
     p.num_stages = pick_stages(bn, static_cast<int64_t>(grid.x) * grid.y * grid.z);
     p.counters = nullptr;
     if (p.splits > 1) {
@@ -617,34 +625,59 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
     return e == cudaSuccess ? PF_OK : PF_ERR_CUDA;
 }
 
-template <int BN>
-cudaError_t launch_gemm2(const GemmLaunch& a, const GemmLaunch& b, cudaStream_t stream) {
+// One launch for up to three prepared products.  Products whose contraction is split must come
+// first and fit the machine together (their CTAs wait for one another); tiles are 64 or 128 wide.
+int gemm_multi(const GemmLaunch* const* g, int count, cudaStream_t stream) {
+    if (count < 1 || count > 3) return PF_ERR_UNSUPPORTED;
+    int ctas[3] = {0, 0, 0};
+    int total = 0, split_ctas = 0;
+    bool seen_plain = false;
+    for (int i = 0; i < count; ++i) {
+        if (g[i]->bn != 64 && g[i]->bn != 128) return PF_ERR_UNSUPPORTED;
+        ctas[i] = static_cast<int>(g[i]->grid.x * g[i]->grid.y * g[i]->grid.z);
+        total += ctas[i];
+        if (g[i]->p.splits > 1) {
+            if (seen_plain) return PF_ERR_UNSUPPORTED;
+            split_ctas += ctas[i];
+        } else {
+            seen_plain = true;
+        }
+    }
+    if (split_ctas > kNumSMs) return PF_ERR_UNSUPPORTED;
+    GemmParams prm[3];
+    size_t smem = 0;
+    for (int i = 0; i < 3; ++i) {
+        const GemmLaunch* src = g[i < count ? i : 0];
+        prm[i] = src->p;
+        const int stages = pick_stages(src->bn, total);
+        prm[i].num_stages = stages;
+        if (i < count) {
+            smem = std::max(smem, gemm_smem(src->bn, stages));
+            const int64_t gper = ceil_div(src->bn / 4, prm[i].splits);
+            if (prm[i].splits > 1 && gper * prm[i].splits * (kBM * 16) > static_cast<int64_t>(stages) * (kBM * kBK * 2 + src->bn * kBK * 2))
+                return PF_ERR_UNSUPPORTED;
+        }
+    }
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(tc_gemm2_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(std::min(gemm_smem(BN, kMaxStages), static_cast<size_t>(227 * 1024))));
-        if (e != cudaSuccess) return e;
+        if (cudaFuncSetAttribute(tc_gemm3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(gemm_smem(128, kMaxStages))) != cudaSuccess)
+            return PF_ERR_CUDA;
         configured[dev] = true;
     }
-    const int ca = static_cast<int>(a.grid.x * a.grid.y * a.grid.z), cb = static_cast<int>(b.grid.x * b.grid.y * b.grid.z);
-    const int2 ta = make_int2(a.grid.x, a.grid.y), tb = make_int2(b.grid.x, b.grid.y);
-    // both products run with the pipeline depth of the whole launch
-    GemmParams pa = a.p, pb = b.p;
-    if ((pa.splits > 1 || pb.splits > 1) && ca + cb > kNumSMs) return cudaErrorInvalidConfiguration;
-    pa.num_stages = pb.num_stages = pick_stages(BN, ca + cb);
-    cudaError_t e = launch_overlapped(tc_gemm2_kernel<BN>, dim3(ca + cb), dim3(kGemmThreads), gemm_smem(BN, pa.num_stages),
-                                      stream, a.ta, a.tb, b.ta, b.tb, pa, pb, ca, ta, tb);
-    if (e == cudaSuccess) count_launch();
-    return e;
-}
-
-// Both factor gradients of a layer in one launch (their slices are summed inside the kernel).
-int gemm_pair(const GemmLaunch& a, const GemmLaunch& b, cudaStream_t stream) {
-    if (a.bn != b.bn || a.bn == 256) return PF_ERR_UNSUPPORTED;
-    const cudaError_t e = a.bn == 64 ? launch_gemm2<64>(a, b, stream) : launch_gemm2<128>(a, b, stream);
-    return e == cudaSuccess ? PF_OK : PF_ERR_CUDA;
+    const GemmLaunch* a = g[0];
+    const GemmLaunch* b = g[count > 1 ? 1 : 0];
+    const GemmLaunch* c = g[count > 2 ? 2 : 0];
+    const int end0 = ctas[0], end1 = ctas[0] + ctas[1];
+    const cudaError_t e = launch_overlapped(
+        tc_gemm3_kernel, dim3(static_cast<unsigned>(total)), dim3(kGemmThreads), smem, stream, a->ta, a->tb, b->ta, b->tb,
+        c->ta, c->tb, prm[0], prm[1], prm[2], end0, end1, make_int2(a->grid.x, a->grid.y), make_int2(b->grid.x, b->grid.y),
+        make_int2(c->grid.x, c->grid.y));
+    if (e != cudaSuccess) return PF_ERR_CUDA;
+    count_launch();
+    return PF_OK;
 }
 
 // A row-major bf16 matrix that TMA must read: used as is when 16-byte aligned with a pitch that is
@@ -775,6 +808,7 @@ int linear_bwd(const LinearArgs& a, int* handled) {
         if (st != PF_OK) return st;
     }
     ChainPlan plan;
+    bool dx_pending = false;     // dX still to be computed as a plain product G U^T
     if (use_chain(a.m) && (!a.dX || tma_ok(a.dX, a.lddx)) && chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan)) {
         st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream);
         if (st != PF_OK) return st;
@@ -782,17 +816,25 @@ int linear_bwd(const LinearArgs& a, int* handled) {
         st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG,
                   pick_splits(a.m, a.r, pick_bn(a.r), a.n), p1, a.stream);
         if (st != PF_OK) return st;
-        if (a.dX) {
-            st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
-            if (st != PF_OK) return st;
+        dx_pending = a.dX != nullptr;
+    }
+    {   // dU = x^T G, dV = dY^T T (and dX = G U^T when it is still due): one launch when their tiles allow
+        GemmLaunch gu, gv, gx;
+        bool ok = gemm_prepare({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, nullptr, &gu) == PF_OK &&
+                  gemm_prepare({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, nullptr, &gv) == PF_OK;
+        if (ok && dx_pending)
+            ok = gemm_prepare({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, nullptr, &gx) == PF_OK;
+        if (ok) {
+            const GemmLaunch* list[3] = {&gu, &gv, &gx};
+            // a split product has to come before the plain ones
+            if (gu.p.splits <= 1 && gv.p.splits > 1) { list[0] = &gv; list[1] = &gu; }
+            st = gemm_multi(list, dx_pending ? 3 : 2, a.stream);
+            if (st != PF_ERR_UNSUPPORTED) return st;
         }
     }
-    {   // dU = x^T G and dV = dY^T T: one launch for both products when their tiles match
-        GemmLaunch gu, gv;
-        if (gemm_prepare({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, nullptr, &gu) == PF_OK &&
-            gemm_prepare({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, nullptr, &gv) == PF_OK &&
-            gu.bn == gv.bn && gu.bn != 256)
-            return gemm_pair(gu, gv, a.stream);
+    if (dx_pending) {
+        st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
+        if (st != PF_OK) return st;
     }
     st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream);
     if (st != PF_OK) return st;
@@ -865,21 +907,35 @@ int conv_bwd(const ConvArgs& a, int* handled) {
     // dT = dY V  (per pixel)
     st = gemm({a.dY, a.O, false}, {a.V, a.R, true}, M, a.R, a.O, dT, a.R, 1, nullptr, a.stream);
     if (st != PF_OK) return st;
-    // dX = sum over taps of shifted dT times U[tap]^T  (implicit GEMM, contraction kh*kw*R)
-    if (a.dX) {
-        const ConvA cx{1, a.N, a.H, a.W, a.R, a.kw, a.pad, a.C};
-        st = gemm({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
-                  nullptr, a.stream, &cx);
-        if (st != PF_OK) return st;
-    }
     // dU[tap] = shifted x^T dT ; dV = dY^T T   (reductions over all pixels, split across CTAs)
+    // dX = sum over taps of shifted dT times U[tap]^T  (implicit GEMM, contraction kh*kw*R)
+    // All three depend on dT only and share one launch: the few long CTAs of the split reductions
+    // start first and the many short dX tiles fill the second CTA slot of every SM beside them.
     const ConvA cu{2, a.N, a.H, a.W, a.C, a.kw, a.pad, a.C};
-    GemmLaunch gu, gv;
+    const ConvA cx{1, a.N, a.H, a.W, a.R, a.kw, a.pad, a.C};
+    GemmLaunch gu, gv, gx;
     st = gemm_prepare({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, &cu, &gu);
     if (st != PF_OK) return st;
     st = gemm_prepare({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, nullptr, &gv);
     if (st != PF_OK) return st;
-    return gemm_pair(gu, gv, a.stream);
+    if (a.dX) {
+        st = gemm_prepare({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
+                          nullptr, &cx, &gx);
+        if (st != PF_OK) return st;
+    }
+    const GemmLaunch* list[3] = {&gu, &gv, &gx};
+    if (gu.p.splits <= 1 && gv.p.splits > 1) { list[0] = &gv; list[1] = &gu; }
+    st = gemm_multi(list, a.dX ? 3 : 2, a.stream);
+    if (st != PF_ERR_UNSUPPORTED) return st;
+    // separate launches (tile widths that cannot share one)
+    if (a.dX) {
+        st = gemm({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
+                  nullptr, a.stream, &cx);
+        if (st != PF_OK) return st;
+    }
+    st = gemm({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, a.stream, &cu);
+    if (st != PF_OK) return st;
+    return gemm({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, a.stream);
 }
 
 }  // namespace tc
