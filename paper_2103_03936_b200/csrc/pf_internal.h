@@ -77,6 +77,16 @@ cudaError_t splitk_reduce2_bf16(const float* pa, void* Ca, int64_t ldca, int64_t
 cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t ld_dst,
                              int64_t rows, int64_t cols, int64_t cols_padded, cudaStream_t stream);
 
+// Several such copies in one launch (row counts and widths below 2^31).
+struct RepackJob {
+    const void* src;
+    int64_t ld_src;
+    void* dst;
+    int64_t ld_dst;
+    int64_t rows, cols, cols_padded;
+};
+cudaError_t repack_rows_bf16_multi(const RepackJob* jobs, int count, cudaStream_t stream);
+
 // pack
 cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const int64_t* offsets,
                         int count, int elem_bytes, void* flat, cudaStream_t stream);

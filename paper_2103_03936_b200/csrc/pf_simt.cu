@@ -238,6 +238,43 @@ repack_rows_kernel(const unsigned short* __restrict__ src, int64_t ld_src,
     }
 }
 
+// Several re-pitch copies in one launch.  A work item is one 16-byte piece (8 elements) of a
+// destination row: the destination is 16-byte aligned with a pitch that is a multiple of 8
+// elements, the source may start anywhere, so it is read element by element.
+constexpr int kRepackJobs = 6;
+struct RepackBatchArgs {
+    const unsigned short* src[kRepackJobs];
+    unsigned short* dst[kRepackJobs];
+    long long ld_src[kRepackJobs], ld_dst[kRepackJobs];
+    int cols[kRepackJobs], pieces_per_row[kRepackJobs];
+    long long item_end[kRepackJobs];   // running total of items up to and including job j
+    int count;
+};
+__global__ void __launch_bounds__(256)
+repack_multi_kernel(const RepackBatchArgs a) {
+    const long long total = a.item_end[a.count - 1];
+    for (long long it = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; it < total;
+         it += static_cast<long long>(gridDim.x) * blockDim.x) {
+        int j = 0;
+        while (j + 1 < a.count && it >= a.item_end[j]) ++j;
+        const long long local = it - (j > 0 ? a.item_end[j - 1] : 0);
+        const int ppr = a.pieces_per_row[j];
+        const long long row = local / ppr;
+        const int c0 = static_cast<int>(local - row * ppr) * 8;
+        const unsigned short* sp = a.src[j] + row * a.ld_src[j] + c0;
+        const int left = a.cols[j] - c0;
+        unsigned short v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = e < left ? sp[e] : static_cast<unsigned short>(0);
+        uint4 o;
+        o.x = v[0] | (static_cast<unsigned int>(v[1]) << 16);
+        o.y = v[2] | (static_cast<unsigned int>(v[3]) << 16);
+        o.z = v[4] | (static_cast<unsigned int>(v[5]) << 16);
+        o.w = v[6] | (static_cast<unsigned int>(v[7]) << 16);
+        *reinterpret_cast<uint4*>(a.dst[j] + row * a.ld_dst[j] + c0) = o;
+    }
+}
+
 }  // namespace
 
 int simt_pick_splits(int64_t M, int64_t N, int64_t K) {
@@ -299,6 +336,48 @@ cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t
                                                    cols_padded);
     count_launch();
     return cudaGetLastError();
+}
+
+cudaError_t repack_rows_bf16_multi(const RepackJob* jobs, int count, cudaStream_t stream) {
+    while (count > 0) {
+        RepackBatchArgs a;
+        a.count = 0;
+        long long total = 0;
+        const int n = count < kRepackJobs ? count : kRepackJobs;
+        for (int i = 0; i < n; ++i) {
+            const RepackJob& j = jobs[i];
+            if (j.rows <= 0 || j.cols <= 0) continue;
+            const bool fast = (reinterpret_cast<uintptr_t>(j.dst) & 15) == 0 && j.ld_dst % 8 == 0 &&
+                              j.cols_padded == (j.cols + 7) / 8 * 8 && j.cols_padded <= j.ld_dst;
+            if (!fast) {   // arbitrary destination: the element-wise copy
+                cudaError_t e = repack_rows_bf16(j.src, j.ld_src, j.dst, j.ld_dst, j.rows, j.cols, j.cols_padded, stream);
+                if (e != cudaSuccess) return e;
+                continue;
+            }
+            const int k = a.count++;
+            a.src[k] = static_cast<const unsigned short*>(j.src);
+            a.dst[k] = static_cast<unsigned short*>(j.dst);
+            a.ld_src[k] = j.ld_src; a.ld_dst[k] = j.ld_dst;
+            a.cols[k] = static_cast<int>(j.cols);
+            a.pieces_per_row[k] = static_cast<int>(j.cols_padded / 8);
+            total += j.rows * (j.cols_padded / 8);
+            a.item_end[k] = total;
+        }
+        if (a.count > 0) {
+            for (int k = a.count; k < kRepackJobs; ++k) {
+                a.src[k] = a.src[0]; a.dst[k] = a.dst[0]; a.ld_src[k] = 0; a.ld_dst[k] = 0; a.cols[k] = 0;
+                a.pieces_per_row[k] = 1; a.item_end[k] = total;
+            }
+            const long long blocks = ceil_div(total, 256) < 8 * kNumSMs ? ceil_div(total, 256) : 8 * kNumSMs;
+            repack_multi_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(a);
+            count_launch();
+            cudaError_t e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+        }
+        jobs += n;
+        count -= n;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace pf

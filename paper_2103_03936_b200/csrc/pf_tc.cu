@@ -688,13 +688,23 @@ struct Staged {
 };
 int64_t pad8(int64_t v) { return (v + 7) / 8 * 8; }
 
+// The re-pitch copies of one call are collected and issued as one launch.
+struct RepackList {
+    RepackJob jobs[6];
+    int count = 0;
+    int flush(cudaStream_t stream) {
+        const cudaError_t e = count > 0 ? repack_rows_bf16_multi(jobs, count, stream) : cudaSuccess;
+        count = 0;
+        return e == cudaSuccess ? PF_OK : PF_ERR_CUDA;
+    }
+};
+
 // returns 0 = usable, 1 = needs repack but no room reserved (decline), <0 never
-int stage_operand(const void* p, int64_t ld, int64_t rows, int64_t cols, char*& scratch, Staged* out,
-                  cudaStream_t stream, int* status) {
+int stage_operand(const void* p, int64_t ld, int64_t rows, int64_t cols, char*& scratch, Staged* out, RepackList* list) {
     if (tma_ok(p, ld)) { out->p = p; out->ld = ld; return 0; }
     if (cols % 8 == 0) return 1;   // the workspace query reserves repack room only for ragged widths
     const int64_t ldp = pad8(cols);
-    if (repack_rows_bf16(p, ld, scratch, ldp, rows, cols, ldp, stream) != cudaSuccess) { *status = PF_ERR_CUDA; return 0; }
+    list->jobs[list->count++] = RepackJob{p, ld, scratch, ldp, rows, cols, ldp};
     out->p = scratch; out->ld = ldp;
     scratch += align_up(static_cast<size_t>(rows) * ldp * 2, 256);
     return 0;
@@ -734,9 +744,11 @@ int linear_fwd(const LinearArgs& a, int* handled) {
     int st = PF_OK;
     char* scratch = a.ws;
     Staged x, U, V;
-    if (stage_operand(a.x, a.ldx, a.m, a.k, scratch, &x, a.stream, &st)) return PF_OK;
-    if (stage_operand(a.U, a.ldu, a.k, a.r, scratch, &U, a.stream, &st)) return PF_OK;
-    if (stage_operand(a.V, a.ldv, a.n, a.r, scratch, &V, a.stream, &st)) return PF_OK;
+    RepackList repacks;
+    if (stage_operand(a.x, a.ldx, a.m, a.k, scratch, &x, &repacks)) return PF_OK;
+    if (stage_operand(a.U, a.ldu, a.k, a.r, scratch, &U, &repacks)) return PF_OK;
+    if (stage_operand(a.V, a.ldv, a.n, a.r, scratch, &V, &repacks)) return PF_OK;
+    st = repacks.flush(a.stream);
     if (st != PF_OK) return st;
     *handled = 1;
     // T: written straight into the stash when TMA can read it back, else into padded scratch
@@ -769,22 +781,23 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     int st = PF_OK;
     char* scratch = a.ws;
     Staged x, U, V, dY, T;
-    if (stage_operand(a.x, a.ldx, a.m, a.k, scratch, &x, a.stream, &st)) return PF_OK;
-    if (stage_operand(a.U, a.ldu, a.k, a.r, scratch, &U, a.stream, &st)) return PF_OK;
-    if (stage_operand(a.V, a.ldv, a.n, a.r, scratch, &V, a.stream, &st)) return PF_OK;
-    if (stage_operand(a.dY, a.lddy, a.m, a.n, scratch, &dY, a.stream, &st)) return PF_OK;
-    if (st != PF_OK) return st;
+    RepackList repacks;
+    if (stage_operand(a.x, a.ldx, a.m, a.k, scratch, &x, &repacks)) return PF_OK;
+    if (stage_operand(a.U, a.ldu, a.k, a.r, scratch, &U, &repacks)) return PF_OK;
+    if (stage_operand(a.V, a.ldv, a.n, a.r, scratch, &V, &repacks)) return PF_OK;
+    if (stage_operand(a.dY, a.lddy, a.m, a.n, scratch, &dY, &repacks)) return PF_OK;
     char* Tbuf = scratch;
     scratch += align_up(static_cast<size_t>(a.m) * pad8(a.r) * 2, 256);
     if (a.T) {
         if (tma_ok(a.T, a.ldt)) { T.p = a.T; T.ld = a.ldt; }
         else if (a.r % 8 == 0) return PF_OK;   // odd pitch on an even width: FMA path
         else {
-            if (repack_rows_bf16(a.T, a.ldt, Tbuf, pad8(a.r), a.m, a.r, pad8(a.r), a.stream) != cudaSuccess)
-                return PF_ERR_CUDA;
+            repacks.jobs[repacks.count++] = RepackJob{a.T, a.ldt, Tbuf, pad8(a.r), a.m, a.r, pad8(a.r)};
             T.p = Tbuf; T.ld = pad8(a.r);
         }
     }
+    st = repacks.flush(a.stream);
+    if (st != PF_OK) return st;
     *handled = 1;
     bool need_T = false;
     if (!a.T) {
