@@ -139,6 +139,26 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     if (warp == 0) {
         if (elect_one()) {
             uint32_t s = 0, ph = 0;
+            // convolution operands: tap / block / image positions advance as counters (an integer
+            // division per k-block would sit on the producer's critical path)
+            int c1_rb = 0, c1_ta = 0, c1_tb = 0, c1_img = 0, c1_h0 = 0;     // conv_mode 1
+            int c2_c0 = 0, c2_x = 0, c2_y = 0, c2_img = 0, c2_t = 0;          // conv_mode 2
+            if (p.conv_mode == 1) {
+                const int tap = kb_beg / p.cv_blks;
+                c1_rb = kb_beg - tap * p.cv_blks;
+                c1_ta = tap / p.cv_kw;
+                c1_tb = tap - c1_ta * p.cv_kw;
+                c1_img = bx / p.cv_tpi;
+                c1_h0 = (bx - c1_img * p.cv_tpi) * p.cv_box_h + p.cv_pad;
+            } else if (p.conv_mode == 2) {
+                const int tap = m0 / p.cv_C;
+                c2_c0 = m0 - tap * p.cv_C;
+                const int ta = tap / p.cv_kw;
+                c2_x = tap - ta * p.cv_kw - p.cv_pad;
+                c2_y = ta - p.cv_pad;
+                c2_img = kb_beg / p.cv_tpi;
+                c2_t = kb_beg - c2_img * p.cv_tpi;
+            }
             for (int i = 0; i < nkb; ++i) {
                 if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag, p.status)) break;
                 const uint32_t full = smem_u32(&ctl->full[s]);
@@ -149,26 +169,23 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                                                         : kStageBytes);
                 const int k0 = (kb_beg + i) * kBK;
                 if (p.conv_mode == 1) {
-                    const int kbg = kb_beg + i;
-                    const int tap = kbg / p.cv_blks, rb = kbg - tap * p.cv_blks;
-                    const int ta = tap / p.cv_kw, tb = tap - ta * p.cv_kw;
-                    const int img = bx / p.cv_tpi;
-                    const int h0 = (bx - img * p.cv_tpi) * p.cv_box_h;
-                    tma_load_4d(a_dst, &tmA, full, rb * 64, p.cv_pad - tb, h0 + p.cv_pad - ta, img);
-                    tma_load_2d(b_dst, &tmB, full, rb * 64, tap * p.cv_C + n0);
+                    tma_load_4d(a_dst, &tmA, full, c1_rb * 64, p.cv_pad - c1_tb, c1_h0 - c1_ta, c1_img);
+                    tma_load_2d(b_dst, &tmB, full, c1_rb * 64, (c1_ta * p.cv_kw + c1_tb) * p.cv_C + n0);
+                    if (++c1_rb == p.cv_blks) {
+                        c1_rb = 0;
+                        if (++c1_tb == p.cv_kw) { c1_tb = 0; ++c1_ta; }
+                    }
                     if (++s == NS) { s = 0; ph ^= 1u; }
                     continue;
                 }
                 if (p.conv_mode == 2) {
-                    const int kbg = kb_beg + i;
-                    const int tap = m0 / p.cv_C, c0 = m0 - tap * p.cv_C;
-                    const int ta = tap / p.cv_kw, tb = tap - ta * p.cv_kw;
-                    const int img = kbg / p.cv_tpi;
-                    const int h0 = (kbg - img * p.cv_tpi) * p.cv_box_h;
-                    tma_load_4d(a_dst, &tmA, full, c0, tb - p.cv_pad, h0 + ta - p.cv_pad, img);
-                    tma_load_4d(a_dst + 8192, &tmA, full, c0 + 64, tb - p.cv_pad, h0 + ta - p.cv_pad, img);
+                    const int hy = c2_t * p.cv_box_h + c2_y;
+                    tma_load_4d(a_dst, &tmA, full, c2_c0, c2_x, hy, c2_img);
+                    tma_load_4d(a_dst + 8192, &tmA, full, c2_c0 + 64, c2_x, hy, c2_img);
 #pragma unroll
-                    for (int h = 0; h < BN / 64; ++h) tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, kbg * p.kpix);
+                    for (int h = 0; h < BN / 64; ++h)
+                        tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, (kb_beg + i) * p.kpix);
+                    if (++c2_t == p.cv_tpi) { c2_t = 0; ++c2_img; }
                     if (++s == NS) { s = 0; ph ^= 1u; }
                     continue;
                 } else if (p.a_mn) {

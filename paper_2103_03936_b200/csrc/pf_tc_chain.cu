@@ -145,6 +145,11 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int q = 0; q < nkb2; ++q) tma_prefetch_l2_2d(&tmB2, q * 64, n0);
             }
             const uint32_t tx1 = static_cast<uint32_t>(p.rows_tile) * 128u + static_cast<uint32_t>(p.r_pad) * 128u;
+            // convolution: (tap row, tap column, channel block) advance as counters; integer divisions
+            // in this loop would sit on the producer's critical path
+            const int cv_img = p.conv_cblks > 0 ? static_cast<int>(blockIdx.x) / p.conv_tiles_per_img : 0;
+            const int cv_h0 = (static_cast<int>(blockIdx.x) - cv_img * p.conv_tiles_per_img) * p.conv_box_h - p.conv_pad;
+            int cv_cb = 0, cv_ta = 0, cv_tb = 0;
             for (int kb = 0; kb < nkb1; ++kb) {
                 ok = mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status);
                 if (!ok) break;
@@ -152,11 +157,11 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const uint32_t dst = ring + rp.off;
                 mbar_expect_tx(full, tx1);
                 if (p.conv_cblks > 0) {
-                    const int tap = kb / p.conv_cblks, cb = kb - tap * p.conv_cblks;
-                    const int ta = tap / p.conv_kw, tb = tap - ta * p.conv_kw;
-                    const int img = static_cast<int>(blockIdx.x) / p.conv_tiles_per_img;
-                    const int h0 = (static_cast<int>(blockIdx.x) - img * p.conv_tiles_per_img) * p.conv_box_h;
-                    tma_load_4d(dst, &tmA, full, cb * 64, tb - p.conv_pad, h0 + ta - p.conv_pad, img);
+                    tma_load_4d(dst, &tmA, full, cv_cb * 64, cv_tb - p.conv_pad, cv_h0 + cv_ta, cv_img);
+                    if (++cv_cb == p.conv_cblks) {
+                        cv_cb = 0;
+                        if (++cv_tb == p.conv_kw) { cv_tb = 0; ++cv_ta; }
+                    }
                 } else {
                     tma_load_2d(dst, &tmA, full, kb * 64, m0);
                 }
