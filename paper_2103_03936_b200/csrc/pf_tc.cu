@@ -6,8 +6,8 @@
 //                       (row-major operands read either along or across the contraction index,
 //                       i.e. K-major or MN-major shared-memory descriptors), with an optional
 //                       reduction split whose fp32 partials are summed in a fixed order.
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..5 = epilogue
-// (each owns the 32 TMEM lanes of its warp-id quadrant).
+// Warp roles: warp 0 = TMA producer of operand A, warp 1 = TMEM allocation + MMA issue, warps 2..5 =
+// epilogue (each owns the 32 TMEM lanes of its warp-id quadrant), warp 6 = TMA producer of operand B.
 #include "pf_tc.h"
 
 #include <cuda.h>
@@ -25,7 +25,7 @@ namespace {
 constexpr int kBM = 128;       // rows of the output tile = TMEM lanes
 constexpr int kBK = 64;        // contraction elements per pipeline stage (128 bytes of bf16)
 constexpr int kMaxStages = 6;
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 224;   // A producer, MMA issue, 4 epilogue warps, B producer
 constexpr int kFixSlots = 32;  // counter sets handed out round-robin to launches that split a contraction
 constexpr int kFixTiles = 160; // output tiles of one split product (tiles * slices never exceeds the SM count)
 
@@ -105,7 +105,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < NS; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->full[s]), 2);     // one expect_tx arrival per producer thread
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->tmem_full), 1);
@@ -134,10 +134,18 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     pdl_launch_dependents();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    // Producer and MMA issuer are each one thread chosen with elect.sync that runs its whole role
+    // Producers and MMA issuer are each one thread chosen with elect.sync that runs its whole role
     // (a thread singled out by a lane-id test issues TMA / tcgen05 instructions several times slower).
-    if (warp == 0) {
+    // Two producers, one per operand: a producer thread needs about 130 ns per stage for its loop,
+    // barrier wait and expect_tx plus 40 ns per TMA instruction, which with four tile loads per
+    // stage paced the whole pipeline when one thread issued both operands.
+    if (warp == 0 || warp == 6) {
         if (elect_one()) {
+            const bool do_a = warp == 0;
+            const uint32_t my_bytes = !do_a ? kBBytes
+                                      : p.conv_mode == 1 ? static_cast<uint32_t>(p.rows_tile) * 128u
+                                      : p.conv_mode == 2 ? static_cast<uint32_t>(p.kpix) * 256u
+                                                         : kABytes;
             uint32_t s = 0, ph = 0;
             // convolution operands: tap / block / image positions advance as counters (an integer
             // division per k-block would sit on the producer's critical path)
@@ -164,13 +172,11 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                 const uint32_t full = smem_u32(&ctl->full[s]);
                 const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
                 const uint32_t b_dst = a_dst + kABytes;
-                mbar_expect_tx(full, p.conv_mode == 1 ? static_cast<uint32_t>(p.rows_tile) * 128u + kBBytes
-                                     : p.conv_mode == 2 ? static_cast<uint32_t>(p.kpix) * 256u + kBBytes
-                                                        : kStageBytes);
+                mbar_expect_tx(full, my_bytes);
                 const int k0 = (kb_beg + i) * kBK;
                 if (p.conv_mode == 1) {
-                    tma_load_4d(a_dst, &tmA, full, c1_rb * 64, p.cv_pad - c1_tb, c1_h0 - c1_ta, c1_img);
-                    tma_load_2d(b_dst, &tmB, full, c1_rb * 64, (c1_ta * p.cv_kw + c1_tb) * p.cv_C + n0);
+                    if (do_a) tma_load_4d(a_dst, &tmA, full, c1_rb * 64, p.cv_pad - c1_tb, c1_h0 - c1_ta, c1_img);
+                    else tma_load_2d(b_dst, &tmB, full, c1_rb * 64, (c1_ta * p.cv_kw + c1_tb) * p.cv_C + n0);
                     if (++c1_rb == p.cv_blks) {
                         c1_rb = 0;
                         if (++c1_tb == p.cv_kw) { c1_tb = 0; ++c1_ta; }
@@ -180,21 +186,25 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                 }
                 if (p.conv_mode == 2) {
                     const int hy = c2_t * p.cv_box_h + c2_y;
-                    tma_load_4d(a_dst, &tmA, full, c2_c0, c2_x, hy, c2_img);
-                    tma_load_4d(a_dst + 8192, &tmA, full, c2_c0 + 64, c2_x, hy, c2_img);
+                    if (do_a) {
+                        tma_load_4d(a_dst, &tmA, full, c2_c0, c2_x, hy, c2_img);
+                        tma_load_4d(a_dst + 8192, &tmA, full, c2_c0 + 64, c2_x, hy, c2_img);
+                    } else {
 #pragma unroll
-                    for (int h = 0; h < BN / 64; ++h)
-                        tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, (kb_beg + i) * p.kpix);
+                        for (int h = 0; h < BN / 64; ++h)
+                            tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, (kb_beg + i) * p.kpix);
+                    }
                     if (++c2_t == p.cv_tpi) { c2_t = 0; ++c2_img; }
                     if (++s == NS) { s = 0; ph ^= 1u; }
                     continue;
-                } else if (p.a_mn) {
-                    tma_load_2d(a_dst, &tmA, full, m0, k0);
-                    tma_load_2d(a_dst + 8192, &tmA, full, m0 + 64, k0);
-                } else {
-                    tma_load_2d(a_dst, &tmA, full, k0, m0);
-                }
-                if (p.b_mn) {
+                } else if (do_a) {
+                    if (p.a_mn) {
+                        tma_load_2d(a_dst, &tmA, full, m0, k0);
+                        tma_load_2d(a_dst + 8192, &tmA, full, m0 + 64, k0);
+                    } else {
+                        tma_load_2d(a_dst, &tmA, full, k0, m0);
+                    }
+                } else if (p.b_mn) {
 #pragma unroll
                     for (int h = 0; h < BN / 64; ++h) tma_load_2d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, k0);
                 } else {
@@ -229,7 +239,7 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
             }
             if (ok) tc_commit(smem_u32(&ctl->tmem_full));
         }
-    } else {
+    } else if (warp < 6) {
         const int q = warp & 3;                          // TMEM lane quadrant this warp may access
         const bool ok = mbar_wait_warp(smem_u32(&ctl->tmem_full), 0, abort_flag, p.status);
         tc_fence_after();
