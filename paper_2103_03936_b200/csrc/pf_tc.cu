@@ -581,8 +581,9 @@ struct GemmLaunch {
 int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
                  int splits, float* partial, const ConvA* cv, GemmLaunch* out) {
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
-    // wide outputs that would need more than one wave of 128-column tiles take 256-column tiles
-    const int bn = (splits <= 1 && N >= 512 && ceil_div(M, kBM) * ceil_div(N, 128) > kNumSMs) ? 256 : pick_bn(N);
+    // wide outputs that would need more than one wave of 128-column tiles (two CTAs per SM) take
+    // 256-column tiles
+    const int bn = (splits <= 1 && N >= 512 && ceil_div(M, kBM) * ceil_div(N, 128) > 2 * kNumSMs) ? 256 : pick_bn(N);
     CUtensorMap& ta = out->ta;
     CUtensorMap& tb = out->tb;
     bool oka, okb;

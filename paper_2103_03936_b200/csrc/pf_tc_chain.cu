@@ -30,7 +30,7 @@ namespace tc {
 namespace {
 
 constexpr int kMaxStages = 8;
-constexpr int kChainThreads = 320;          // producer warp, MMA warp, 8 epilogue warps
+constexpr int kChainThreads = 352;          // A producer, MMA warp, 8 epilogue warps, B producer
 constexpr uint32_t kTileBytes = 16384;      // 128 rows x 64 bf16
 constexpr int kAccBufs = 4;                 // 4 x 128 TMEM columns of phase-2 accumulators
 
@@ -103,7 +103,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < NS; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->full[s]), 2);     // one arrival per producer thread
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->t_full), 1);
@@ -135,27 +135,19 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // loops below carry running offsets instead of recomputing them.)
     if (warp == 0) {
         if (elect_one()) {
-            // -------------------------------------------------------------- TMA producer
+            // -------------------------------------------------------------- TMA producer of A (phase 1)
             RingPos rp;
-            bool ok = true;
-            // Phase 2 streams B2 tiles that nobody has touched yet; have L2 fetch them while phase 1
-            // runs.  The CTAs that share these tiles each ask for a different one.
-            if (ntile > 0) {
-                const int n0 = (t_beg + static_cast<int>(blockIdx.x) % ntile) * 128;
-                for (int q = 0; q < nkb2; ++q) tma_prefetch_l2_2d(&tmB2, q * 64, n0);
-            }
-            const uint32_t tx1 = static_cast<uint32_t>(p.rows_tile) * 128u + static_cast<uint32_t>(p.r_pad) * 128u;
+            const uint32_t txa = static_cast<uint32_t>(p.rows_tile) * 128u;
             // convolution: (tap row, tap column, channel block) advance as counters; integer divisions
             // in this loop would sit on the producer's critical path
             const int cv_img = p.conv_cblks > 0 ? static_cast<int>(blockIdx.x) / p.conv_tiles_per_img : 0;
             const int cv_h0 = (static_cast<int>(blockIdx.x) - cv_img * p.conv_tiles_per_img) * p.conv_box_h - p.conv_pad;
             int cv_cb = 0, cv_ta = 0, cv_tb = 0;
             for (int kb = 0; kb < nkb1; ++kb) {
-                ok = mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status);
-                if (!ok) break;
+                if (!mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status)) break;
                 const uint32_t full = full0 + 8 * rp.s;
                 const uint32_t dst = ring + rp.off;
-                mbar_expect_tx(full, tx1);
+                mbar_expect_tx(full, txa);
                 if (p.conv_cblks > 0) {
                     tma_load_4d(dst, &tmA, full, cv_cb * 64, cv_tb - p.conv_pad, cv_h0 + cv_ta, cv_img);
                     if (++cv_cb == p.conv_cblks) {
@@ -165,8 +157,30 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 } else {
                     tma_load_2d(dst, &tmA, full, kb * 64, m0);
                 }
-                for (int q = 0; q < nkb2; ++q)
-                    tma_load_2d(dst + kTileBytes + q * 8192, &tmB1, full, q * 64, kb * 64);
+                rp.advance(NS, S);
+            }
+        }
+    } else if (warp == 10) {
+        if (elect_one()) {
+            // -------------------------------------------------------------- TMA producer of B1 and B2
+            // (a second thread: a producer spends about 130 ns per stage on its loop, barrier wait and
+            // expect_tx and 40 ns per TMA instruction, which paced phase 1 when one thread issued both)
+            RingPos rp;
+            bool ok = true;
+            // Phase 2 streams B2 tiles that nobody has touched yet; have L2 fetch them while phase 1
+            // runs.  The CTAs that share these tiles each ask for a different one.
+            if (ntile > 0) {
+                const int n0 = (t_beg + static_cast<int>(blockIdx.x) % ntile) * 128;
+                for (int q = 0; q < nkb2; ++q) tma_prefetch_l2_2d(&tmB2, q * 64, n0);
+            }
+            const uint32_t txb = static_cast<uint32_t>(p.r_pad) * 128u;
+            for (int kb = 0; kb < nkb1; ++kb) {
+                ok = mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status);
+                if (!ok) break;
+                const uint32_t full = full0 + 8 * rp.s;
+                const uint32_t dst = ring + rp.off + kTileBytes;
+                mbar_expect_tx(full, txb);
+                for (int q = 0; q < nkb2; ++q) tma_load_2d(dst + q * 8192, &tmB1, full, q * 64, kb * 64);
                 rp.advance(NS, S);
             }
             for (int j = 0; j < ntile && ok; ++j) {
@@ -176,6 +190,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     ok = mbar_wait(empty0 + 8 * rp.s, rp.ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
                     const uint32_t full = full0 + 8 * rp.s;
+                    mbar_arrive(full);                      // stands in for the A producer, idle in phase 2
                     mbar_expect_tx(full, kTileBytes * nb);
                     for (int q = 0; q < nb; ++q)
                         tma_load_2d(ring + rp.off + q * kTileBytes, &tmB2, full, (kb + q) * 64, n0);
@@ -253,7 +268,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
             if (stash) tma_store_wait_read<0>();
         }
-    } else {
+    } else if (warp < 10) {
         // ------------------------------------------------------------------ epilogue warps
         // Eight warps: warp w may touch the TMEM lanes of quadrant w % 4, so two warps share each
         // 32-row quadrant and split the columns (64 of every 128) between them.
