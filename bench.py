@@ -310,8 +310,11 @@ def run_ours(args):
     launches0 = pf.pf_launch_count()
 
     def timed_step(i):
+        # the dominant kernel's launch is bracketed by events on every eighth step only: the two
+        # event records end the overlap of consecutive kernels and cost about 5 us per bracket
+        sample = (i % 8) == 0
         for name, call in w.calls[i % NSETS]:
-            if name == dom_name:
+            if name == dom_name and sample:
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record()
                 call()

@@ -117,6 +117,19 @@ def test_configs_full_size_sampled(name, imgs):
     assert pf.pf_last_device_status() == 0
 
 
+def test_backward_is_bit_reproducible():
+    """dU and dV are sums over all pixels split across CTAs; the slices are added in a fixed order."""
+    c = wl.ConvCase("rep", 8, 32, 32, 128, 64, 128, wl.BF16, 31)
+    d = c.generate()
+    x, U, V, dY = (dev(d[k_], wl.BF16) for k_ in ("x", "U", "V", "dY"))
+    a = pf.pf_lowrank_conv_bwd(x, U, V, dY)
+    b = pf.pf_lowrank_conv_bwd(x, U, V, dY)
+    torch.cuda.synchronize()
+    for p, q in zip(a, b):
+        assert torch.equal(p, q)
+    assert pf.pf_last_device_status() == 0
+
+
 def test_empty_batch():
     x = torch.empty((0, 8, 8, 8), dtype=torch.bfloat16, device="cuda")
     U = torch.ones((3, 3, 8, 4), dtype=torch.bfloat16, device="cuda")

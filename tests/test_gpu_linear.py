@@ -169,6 +169,30 @@ def test_backward_is_bit_reproducible(dtype):
         assert torch.equal(p, q)
 
 
+def test_split_reductions_on_two_streams_do_not_interfere():
+    """The slice sums of dU / dV meet at per-tile counters inside the library; launches that are in
+    flight at the same time on different streams must use different counter sets."""
+    cases = [wl.LinearCase("s0", 4096, 256, 320, 64, wl.BF16, 21), wl.LinearCase("s1", 3000, 384, 256, 128, wl.BF16, 22)]
+    ins = []
+    for c in cases:
+        d = c.generate()
+        ins.append(tuple(dev(d[k_], wl.BF16) for k_ in ("x", "U", "V", "dY")))
+    ref = [pf.pf_lowrank_linear_bwd(*t) for t in ins]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[], []]
+    for it in range(6):
+        for i, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                outs[i].append(pf.pf_lowrank_linear_bwd(*ins[i], stream=st))
+    torch.cuda.synchronize()
+    for i in range(2):
+        for got in outs[i]:
+            for p, q in zip(got, ref[i]):
+                assert torch.equal(p, q)
+    assert pf.pf_last_device_status() == 0
+
+
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_empty_batch(dtype):
     tdt = torch.float32 if dtype == wl.F32 else torch.bfloat16
