@@ -68,11 +68,6 @@ int simt_pick_splits(int64_t M, int64_t N, int64_t K);
 cudaError_t splitk_reduce(const float* partial, void* C, int64_t ldc, int64_t M, int64_t N, int splits,
                           int dtype, cudaStream_t stream);
 
-// Two bf16 split reductions in one launch (falls back to two launches for odd shapes).
-cudaError_t splitk_reduce2_bf16(const float* pa, void* Ca, int64_t ldca, int64_t Ma, int64_t Na, int sa,
-                                const float* pb, void* Cb, int64_t ldcb, int64_t Mb, int64_t Nb, int sb,
-                                cudaStream_t stream);
-
 // Strided 2-D copy with zero fill (repack to a padded pitch), elements of 2 bytes.
 cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t ld_dst,
                              int64_t rows, int64_t cols, int64_t cols_padded, cudaStream_t stream);

@@ -17,8 +17,8 @@
 namespace pf {
 namespace {
 
-constexpr int kPackBatch = 96;          // tensors per launch (parameter space is 4 KB)
-constexpr int kVecPerChunk = 1024;      // 16 KB of destination per block-chunk
+constexpr int kPackBatch = 512;         // tensors per launch (the table travels in the kernel parameters: 14 KB of the 32 KB limit)
+constexpr int kVecPerChunk = 512;       // 8 KB of destination per block-chunk
 constexpr int kPackThreads = 256;
 
 struct PackBatch {

@@ -149,55 +149,6 @@ splitk_reduce_kernel(const float* __restrict__ partial, void* C, int64_t ldc, in
     }
 }
 
-// Two independent split reductions (dU and dV of one layer) in one launch.
-struct ReduceJob {
-    const float* partial;
-    void* C;
-    int64_t ldc, M, N;
-    int splits;
-};
-__global__ void __launch_bounds__(256)
-splitk_reduce2_kernel(const ReduceJob a, const ReduceJob b, int blocks_a) {
-    // A block sums 64 consecutive float4 elements; its four 64-thread groups each take every
-    // fourth slice (in increasing order) and the four group sums are then added in group order,
-    // so the association is fixed and the result is bit-reproducible run to run.
-    __shared__ float4 part[3][64];
-    const bool first = static_cast<int>(blockIdx.x) < blocks_a;
-    const ReduceJob& j = first ? a : b;
-    const int64_t blk = first ? blockIdx.x : blockIdx.x - blocks_a;
-    const int64_t total4 = j.M * j.N / 4;           // N % 4 == 0 on this path
-    const int lane64 = threadIdx.x & 63, grp = threadIdx.x >> 6;
-    const int64_t e = blk * 64 + lane64;
-    const float4* src = reinterpret_cast<const float4*>(j.partial);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (e < total4) {
-        for (int z0 = grp; z0 < j.splits; z0 += 16) {
-            float4 t[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                t[u] = (z0 + 4 * u < j.splits) ? __ldcs(src + static_cast<int64_t>(z0 + 4 * u) * total4 + e)
-                                               : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
-        }
-    }
-    if (grp > 0) part[grp - 1][lane64] = acc;
-    __syncthreads();
-    if (grp == 0 && e < total4) {
-#pragma unroll
-        for (int g = 0; g < 3; ++g) {
-            const float4 t = part[g][lane64];
-            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
-        }
-        const int64_t el = e * 4, row = el / j.N, col = el - row * j.N;
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-        uint2 o;
-        o.x = *reinterpret_cast<unsigned int*>(&lo);
-        o.y = *reinterpret_cast<unsigned int*>(&hi);
-        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(j.C) + row * j.ldc + col) = o;
-    }
-}
-
 template <typename T>
 cudaError_t launch_typed(const SimtGemm& g, cudaStream_t stream) {
     dim3 grid(static_cast<unsigned>(ceil_div(g.M, BM)), static_cast<unsigned>(ceil_div(g.N, BN)),
@@ -294,26 +245,6 @@ cudaError_t splitk_reduce(const float* partial, void* C, int64_t ldc, int64_t M,
     const int blocks = static_cast<int>(ceil_div(total, 256) < 4 * kNumSMs ? ceil_div(total, 256) : 4 * kNumSMs);
     if (dtype == PF_BF16) splitk_reduce_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(partial, C, ldc, M, N, splits);
     else splitk_reduce_kernel<float><<<blocks, 256, 0, stream>>>(partial, C, ldc, M, N, splits);
-    cudaError_t e = cudaGetLastError();
-    if (e == cudaSuccess) count_launch();
-    return e;
-}
-
-cudaError_t splitk_reduce2_bf16(const float* pa, void* Ca, int64_t ldca, int64_t Ma, int64_t Na, int sa,
-                                const float* pb, void* Cb, int64_t ldcb, int64_t Mb, int64_t Nb, int sb,
-                                cudaStream_t stream) {
-    const bool vec = Na % 4 == 0 && Nb % 4 == 0 && ldca % 4 == 0 && ldcb % 4 == 0 &&
-                     (reinterpret_cast<uintptr_t>(Ca) & 7) == 0 && (reinterpret_cast<uintptr_t>(Cb) & 7) == 0;
-    if (!vec) {
-        cudaError_t e = splitk_reduce(pa, Ca, ldca, Ma, Na, sa, PF_BF16, stream);
-        if (e != cudaSuccess) return e;
-        return splitk_reduce(pb, Cb, ldcb, Mb, Nb, sb, PF_BF16, stream);
-    }
-    const ReduceJob a{pa, Ca, ldca, Ma, Na, sa}, b{pb, Cb, ldcb, Mb, Nb, sb};
-    auto blocks = [](int64_t M, int64_t N) { return static_cast<int>(ceil_div(M * N / 4, 64)); };
-    if (ceil_div(Ma * Na / 4, 64) + ceil_div(Mb * Nb / 4, 64) > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    const int ba = blocks(Ma, Na), bb = blocks(Mb, Nb);
-    splitk_reduce2_kernel<<<ba + bb, 256, 0, stream>>>(a, b, ba);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) count_launch();
     return e;

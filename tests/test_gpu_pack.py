@@ -56,7 +56,7 @@ def test_c4_factor_gradient_list():
 
 def test_many_tensors_span_several_launches():
     rng = np.random.default_rng(0)
-    numels = [int(v) for v in rng.integers(0, 3000, size=250)]
+    numels = [int(v) for v in rng.integers(0, 3000, size=1100)]   # more than two launches' worth of tensors
     check_pack(numels, wl.BF16, src_shift=[0, 1, 2, 3])
 
 
