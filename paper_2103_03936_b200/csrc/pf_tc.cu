@@ -53,6 +53,8 @@ struct GemmParams {
     int tiles_x;             // row tiles of this product (tile id = column tile * tiles_x + row tile)
     void* C;                 // bf16 [M, ldc]
     long long ldc;
+    void* C2;                // optional second copy of the result at another pitch (split contractions only)
+    long long ldc2;
     float* partial;          // splits > 1: fp32 slices, one 128 x BN block per (tile, slice)
     unsigned int* counters;  // splits > 1: two counters per tile
     unsigned int* status;
@@ -425,6 +427,26 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                 if (col + 3 < p.N) dst[3] = __float2bfloat16_rn(acc.w);
             }
         }
+        if (p.C2) {   // the same sums once more, for a destination whose pitch the first cannot have
+            __nv_bfloat16* C2b = reinterpret_cast<__nv_bfloat16*>(p.C2);
+            for (int id = threadIdx.x; id < ng * kBM; id += kGemmThreads) {
+                const int gl = id / kBM, rr = id % kBM;
+                float4 acc = sm4[id];
+#pragma unroll 8
+                for (int s = 1; s < S; ++s) {
+                    const float4 t = sm4[static_cast<uint32_t>(s) * share4 + static_cast<uint32_t>(id)];
+                    acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+                }
+                const int row = m0 + rr, col = n0 + (g_beg + gl) * 4;
+                if (row < p.M) {
+                    __nv_bfloat16* dst = C2b + static_cast<size_t>(row) * p.ldc2 + col;
+                    if (col < p.N) dst[0] = __float2bfloat16_rn(acc.x);
+                    if (col + 1 < p.N) dst[1] = __float2bfloat16_rn(acc.y);
+                    if (col + 2 < p.N) dst[2] = __float2bfloat16_rn(acc.z);
+                    if (col + 3 < p.N) dst[3] = __float2bfloat16_rn(acc.w);
+                }
+            }
+        }
     }
     __syncthreads();
     if (threadIdx.x == 0 && ctl->fix_ok) {
@@ -602,6 +624,7 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.a_mn = A.mn_major; p.b_mn = B.mn_major;
     p.C = C; p.ldc = ldc; p.partial = partial;
+    p.C2 = nullptr; p.ldc2 = 0;
     p.conv_mode = 0; p.cv_blks = 1; p.cv_kw = 1; p.cv_pad = 0; p.cv_C = 1; p.cv_box_h = 1; p.cv_tpi = 1;
     if (cv) {
         p.conv_mode = cv->mode; p.cv_kw = cv->kw; p.cv_pad = cv->pad; p.cv_C = cv->Cw;
@@ -640,12 +663,20 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     return PF_OK;
 }
 
+// `copy2` (optional): asks for a second copy of C at pitch ldc2; *copy2_done tells whether the launch
+// wrote it (only a split contraction can), else the caller copies C itself.
 int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
-         int splits, float* partial, cudaStream_t stream, const ConvA* cv = nullptr) {
+         int splits, float* partial, cudaStream_t stream, const ConvA* cv = nullptr, void* copy2 = nullptr,
+         int64_t ldc2 = 0, bool* copy2_done = nullptr) {
     GemmLaunch g;
     int st = gemm_prepare(A, B, M, N, K, C, ldc, splits, partial, cv, &g);
     if (st == PF_ERR_UNSUPPORTED && splits > 1) st = gemm_prepare(A, B, M, N, K, C, ldc, 1, nullptr, cv, &g);
     if (st != PF_OK) return st;
+    if (copy2_done) *copy2_done = false;
+    if (copy2 && g.p.splits > 1) {
+        g.p.C2 = copy2; g.p.ldc2 = ldc2;
+        if (copy2_done) *copy2_done = true;
+    }
     const GemmParams& p = g.p;
     cudaError_t e = g.bn == 64    ? launch_gemm<64>(g.ta, g.tb, p, g.grid, stream)
                     : g.bn == 128 ? launch_gemm<128>(g.ta, g.tb, p, g.grid, stream)
@@ -785,6 +816,7 @@ int linear_fwd(const LinearArgs& a, int* handled) {
     const bool stash_direct = a.T && tma_ok(a.T, a.ldt);
     if (stash_direct) { T = a.T; ldT = a.ldt; }
     ChainPlan plan;
+    bool stash_written = false;   // the stash at its own (TMA-unreadable) pitch came out of the first product
     if (use_chain(a.m) && tma_ok(a.y, a.ldy) && chain_plan(a.m, a.k, a.n, a.r, true, &plan)) {
         // one fused kernel; the intermediate leaves the chip only if a stash was asked for
         st = chain(x.p, x.ld, a.m, a.k, U.p, U.ld, a.r, V.p, V.ld, a.n, a.y, a.ldy, a.T ? T : nullptr, ldT,
@@ -792,12 +824,13 @@ int linear_fwd(const LinearArgs& a, int* handled) {
     } else {
         float* p1 = reinterpret_cast<float*>(scratch + align_up(static_cast<size_t>(a.m) * pad8(a.r) * 2, 256));
         st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, T, ldT,
-                  pick_splits(a.m, a.r, pick_bn(a.r), a.k), p1, a.stream);
+                  pick_splits(a.m, a.r, pick_bn(a.r), a.k), p1, a.stream, nullptr,
+                  (a.T && !stash_direct) ? a.T : nullptr, a.ldt, &stash_written);
         if (st != PF_OK) return st;
         st = gemm({T, ldT, false}, {V.p, V.ld, false}, a.m, a.n, a.r, a.y, a.ldy, 1, nullptr, a.stream);
     }
     if (st != PF_OK) return st;
-    if (a.T && !stash_direct &&
+    if (a.T && !stash_direct && !stash_written &&
         repack_rows_bf16(T, ldT, a.T, a.ldt, a.m, a.r, a.r, a.stream) != cudaSuccess)
         return PF_ERR_CUDA;
     return PF_OK;
