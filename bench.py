@@ -40,9 +40,9 @@ NSETS = 4  # activation buffer sets rotated between steps so that inputs never s
 # DRAM read + write bytes of one FFN-up forward launch of the dominant kernel, from the ncu capture
 # summarised in profiles/tc_chain_kernel_ffn_forward.md; valid while the kernel's sources hash to the
 # value recorded with that capture.
-DOMINANT_TRAFFIC_BYTES = 9082880
+DOMINANT_TRAFFIC_BYTES = 9084672
 DOMINANT_SOURCES = ("pf_tc_chain.cu", "pf_tc_prims.cuh", "pf_tc_host.h")
-DOMINANT_SHA256 = "6d4bfcc0957e6fac62cbdee8a775dd7364b8cdd66f05df90003ecf8b6bc50516"
+DOMINANT_SHA256 = "a4c5f485b88c2c08e68028e4b3bcd3fb31d23d698df0a824764a23c60a98e8cb"
 
 
 def dominant_traffic():
