@@ -37,9 +37,9 @@ WORKLOAD = ("Transformer FFN factorized linear bf16: m=8192 (64x128 tokens), 512
             "2048->512 r=128, fwd+bwd (dX,dU,dV) + pf_pack_factor_grads of the 4 factor grads")
 NSETS = 4  # activation buffer sets rotated between steps so that inputs never sit in L2
 
-# DRAM read + write bytes of one FFN-up forward launch of the dominant kernel, from the ncu capture
-# summarised in profiles/tc_chain_kernel_ffn_forward.md; valid while the kernel's sources hash to the
-# value recorded with that capture.
+# DRAM read + write bytes of one FFN-up forward launch of the dominant kernel, from an ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum; its summary is kept with the other profile
+# summaries); valid while the kernel's sources hash to the value recorded with that capture.
 DOMINANT_TRAFFIC_BYTES = 9084672
 DOMINANT_SOURCES = ("pf_tc_chain.cu", "pf_tc_prims.cuh", "pf_tc_host.h")
 DOMINANT_SHA256 = "a4c5f485b88c2c08e68028e4b3bcd3fb31d23d698df0a824764a23c60a98e8cb"
