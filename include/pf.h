@@ -22,6 +22,13 @@
  *   - `workspace` is caller-provided scratch of at least the matching
  *     pf_*_workspace() query, 256-byte aligned; its contents are undefined afterwards.
  *     Two calls that may overlap on the GPU must not share a workspace.
+ *   - Besides the workspace the library keeps a few fixed device arrays of its own (a
+ *     status word and 40 KB of counters at which the thread blocks of a split reduction
+ *     meet); calls on different streams of one device may be in flight together: each
+ *     launch takes the next of 32 counter sets, so do not keep more than 32 backward
+ *     calls of one device unfinished at a time.
+ *   - Gradients that are sums over the batch (dU, dV) are added in a fixed order:
+ *     repeating a call on the same inputs gives bit-identical results.
  *   - Every entry returns a pf_status.  Errors detected on the host (bad pointer,
  *     bad dimension, workspace too small, ...) are returned BEFORE anything is
  *     launched.  Nothing is printed, nothing aborts.
