@@ -668,6 +668,14 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
 int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
          int splits, float* partial, cudaStream_t stream, const ConvA* cv = nullptr, void* copy2 = nullptr,
          int64_t ldc2 = 0, bool* copy2_done = nullptr) {
+    // wide, many-tile (tensor-bound) products run on CTA pairs, which halve the operand traffic per SM
+    if (!cv && splits <= 1 && N >= 256 && ceil_div(M, kBM) * ceil_div(N, 128) > 2 * kNumSMs) {
+        const int st2 = gemm_pair_2sm(A.p, A.ld, A.mn_major, B.p, B.ld, B.mn_major, M, N, K, C, ldc, stream);
+        if (st2 != PF_ERR_UNSUPPORTED) {
+            if (copy2_done) *copy2_done = false;
+            return st2;
+        }
+    }
     GemmLaunch g;
     int st = gemm_prepare(A, B, M, N, K, C, ldc, splits, partial, cv, &g);
     if (st == PF_ERR_UNSUPPORTED && splits > 1) st = gemm_prepare(A, B, M, N, K, C, ldc, 1, nullptr, cv, &g);

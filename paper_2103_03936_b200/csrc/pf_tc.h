@@ -45,6 +45,11 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
           cudaStream_t stream, const ChainConv* conv = nullptr);
 
+// Plain product on CTA pairs (pf_tc_pair.cu); PF_ERR_UNSUPPORTED when the output is not 16-byte aligned
+// with a pitch that is a multiple of 8 elements.
+int gemm_pair_2sm(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, int64_t M, int64_t N,
+                  int64_t K, void* C, int64_t ldc, cudaStream_t stream);
+
 size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool bwd);
 size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
                             int pad, bool bwd);

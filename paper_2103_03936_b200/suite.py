@@ -64,6 +64,33 @@ def _time(calls_per_set, iters, warmup=3, repeats=5):
     return out
 
 
+def _library_linear(sets, U, V, iters):
+    """The paper's structure on the same GPU, for context: two library matmuls forward and four
+    backward through PyTorch (cuBLAS), intermediates in HBM.  Returns (fwd, bwd, fwd+bwd) in us."""
+    calls = []
+    for (x, dY) in sets:
+        m, r, n, k = x.shape[0], U.shape[1], V.shape[0], U.shape[0]
+        T = torch.empty((m, r), dtype=x.dtype, device="cuda")
+        y = torch.empty((m, n), dtype=x.dtype, device="cuda")
+        G = torch.empty((m, r), dtype=x.dtype, device="cuda")
+        dX = torch.empty((m, k), dtype=x.dtype, device="cuda")
+        dU, dV = torch.empty_like(U), torch.empty_like(V)
+
+        def fwd(x=x, T=T, y=y):
+            torch.matmul(x, U, out=T)
+            torch.matmul(T, V.t(), out=y)
+
+        def bwd(x=x, dY=dY, T=T, G=G, dX=dX, dU=dU, dV=dV):
+            torch.matmul(dY, V, out=G)
+            torch.matmul(G, U.t(), out=dX)
+            torch.matmul(x.t(), G, out=dU)
+            torch.matmul(dY.t(), T, out=dV)
+
+        calls.append((fwd, bwd))
+    t = _time(calls, iters)
+    return t[0]["median_us"], t[1]["median_us"], t[-1]["median_us"]
+
+
 def _floors(flops_fwd, bytes_fwd, bytes_bwd, pk):
     f = max(flops_fwd / (pk["bf16_tflops"] * 1e12), bytes_fwd / (pk["hbm_gbs"] * 1e9)) * 1e6
     b = max(2 * flops_fwd / (pk["bf16_tflops"] * 1e12), bytes_bwd / (pk["hbm_gbs"] * 1e9)) * 1e6
@@ -82,8 +109,10 @@ def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32):
     U, V = _rand((k, r), tdt, sig, ld=ldr), _rand((n, r), tdt, sig, ld=ldr)
     stream = torch.cuda.current_stream()
     sets = []
+    lib_sets = []
     for _ in range(nsets):
         x, dY = _rand((m, k), tdt, ld=ldk), _rand((m, n), tdt)
+        lib_sets.append((x, dY))
         y = torch.empty((m, n), dtype=tdt, device="cuda")
         T = _rand((m, r), tdt, ld=ldr)
         dX = _rand((m, k), tdt, ld=ldk)
@@ -104,7 +133,9 @@ def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32):
     bytes_bwd = s * (m * n + 2 * m * k + 2 * r * (k + n))
     ff, fb = _floors(flops_fwd, bytes_fwd, bytes_bwd, pk)
     tot = t[-1]["median_us"]
+    lib = _library_linear(lib_sets, U, V, iters)
     return {"config": name, "kind": "linear", "m": m, "k": k, "n": n, "r": r, "dtype": dtype,
+            "library_fwd_us": lib[0], "library_bwd_us": lib[1], "library_fwd_bwd_us": lib[2],
             "pitch": "padded to 16 B" if pad_pitch else "tight", "buffer_sets": nsets, "launches_fwd_bwd": launches,
             "fwd_us": t[0]["median_us"], "bwd_us": t[1]["median_us"], "fwd_bwd_us": tot,
             "floor_fwd_us": ff, "floor_bwd_us": fb, "roofline_frac": (ff + fb) / tot,

@@ -81,6 +81,13 @@ def test_fused_chain_envelope(m, k, n, r):
     run_case(wl.LinearCase("chain", m, k, n, r, wl.BF16, 14), stash=False, need_dX=False)
 
 
+@pytest.mark.parametrize("m,k,n,r", [(16000, 72, 264, 520), (9000, 200, 520, 392)])
+def test_wide_unfused_products_on_cta_pairs(m, k, n, r):
+    """Ranks above 384 run as plain products; wide ones with many tiles use the two-CTA MMA kernel:
+    a ragged last row pair, ragged column tiles and a ragged k tail, K-major and MN-major B."""
+    run_case(wl.LinearCase("pairs", m, k, n, r, wl.BF16, 17))
+
+
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_leading_dimensions_and_padding_untouched(dtype):
     run_case(wl.LinearCase("ld", 200, 72, 136, 24, dtype, 8), ld_pad=8)
