@@ -565,6 +565,14 @@ int pick_splits(int64_t M, int64_t N, int bn, int64_t K) {
 }
 int pick_bn(int64_t N) { return N <= 64 ? 64 : 128; }
 
+// CTA pairs (256 x 256 tiles, persistent) pay off for wide outputs once every pair gets at least two
+// tiles, or fewer tiles with a long contraction each; short products with few tiles are better
+// off as many small single-CTA tiles.
+bool pair_worthwhile(int64_t M, int64_t N, int64_t K) {
+    const int64_t tiles = ceil_div(M, 256) * ceil_div(N, 256);
+    return N >= 256 && (tiles >= kNumSMs || (tiles >= 48 && K >= 2048));
+}
+
 // Slice counts for two products that share one launch (dU: Mu x N, dV: Mv x N, both contracting
 // over K): all CTAs should fit one wave and finish together, so the longest CTA (in k-blocks) is
 // minimised subject to tiles_u * su + tiles_v * sv <= SM count.
@@ -669,7 +677,7 @@ int gemm(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, vo
          int splits, float* partial, cudaStream_t stream, const ConvA* cv = nullptr, void* copy2 = nullptr,
          int64_t ldc2 = 0, bool* copy2_done = nullptr) {
     // wide, many-tile (tensor-bound) products run on CTA pairs, which halve the operand traffic per SM
-    if (!cv && splits <= 1 && N >= 256 && ceil_div(M, kBM) * ceil_div(N, 128) > 2 * kNumSMs) {
+    if (!cv && splits <= 1 && pair_worthwhile(M, N, K)) {
         const int st2 = gemm_pair_2sm(A.p, A.ld, A.mn_major, B.p, B.ld, B.mn_major, M, N, K, C, ldc, stream);
         if (st2 != PF_ERR_UNSUPPORTED) {
             if (copy2_done) *copy2_done = false;
@@ -776,8 +784,10 @@ int stage_operand(const void* p, int64_t ld, int64_t rows, int64_t cols, char*& 
     scratch += align_up(static_cast<size_t>(rows) * ldp * 2, 256);
     return 0;
 }
-// The fused chain pays off once there are enough 128-row tiles to fill the machine.
-bool use_chain(int64_t m) { return m >= 2048; }
+// The fused chain pays off once there are enough 128-row tiles to fill the machine, and while the
+// rank is small enough for the layer to be bound by memory traffic: from r = 256 up the two
+// products are tensor-bound and run faster unfused on CTA pairs (the intermediate is only m x r).
+bool use_chain(int64_t m, int64_t r) { return m >= 2048 && r <= 192; }
 
 size_t repack_room(int64_t rows, int64_t cols) {
     return cols % 8 == 0 ? 0 : align_up(static_cast<size_t>(rows) * pad8(cols) * 2, 256);
@@ -825,7 +835,7 @@ int linear_fwd(const LinearArgs& a, int* handled) {
     if (stash_direct) { T = a.T; ldT = a.ldt; }
     ChainPlan plan;
     bool stash_written = false;   // the stash at its own (TMA-unreadable) pitch came out of the first product
-    if (use_chain(a.m) && tma_ok(a.y, a.ldy) && chain_plan(a.m, a.k, a.n, a.r, true, &plan)) {
+    if (use_chain(a.m, a.r) && tma_ok(a.y, a.ldy) && chain_plan(a.m, a.k, a.n, a.r, true, &plan)) {
         // one fused kernel; the intermediate leaves the chip only if a stash was asked for
         st = chain(x.p, x.ld, a.m, a.k, U.p, U.ld, a.r, V.p, V.ld, a.n, a.y, a.ldy, a.T ? T : nullptr, ldT,
                    a.stream);
@@ -891,7 +901,7 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     }
     ChainPlan plan;
     bool dx_pending = false;     // dX still to be computed as a plain product G U^T
-    if (use_chain(a.m) && (!a.dX || tma_ok(a.dX, a.lddx)) && chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan)) {
+    if (use_chain(a.m, a.r) && (!a.dX || tma_ok(a.dX, a.lddx)) && chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan)) {
         st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream);
         if (st != PF_OK) return st;
     } else {
@@ -912,6 +922,16 @@ int linear_bwd(const LinearArgs& a, int* handled) {
             if (gu.p.splits <= 1 && gv.p.splits > 1) { list[0] = &gv; list[1] = &gu; }
             st = gemm_multi(list, dx_pending ? 3 : 2, a.stream);
             if (st != PF_ERR_UNSUPPORTED) return st;
+            if (dx_pending) {
+                // dX has wide tiles of its own (CTA pairs): launch it alone, dU and dV still together
+                st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
+                if (st != PF_OK) return st;
+                dx_pending = false;
+                if (!(pair_worthwhile(a.k, a.r, a.m) && pair_worthwhile(a.n, a.r, a.m))) {
+                    st = gemm_multi(list, 2, a.stream);
+                    if (st != PF_ERR_UNSUPPORTED) return st;
+                }
+            }
         }
     }
     if (dx_pending) {
