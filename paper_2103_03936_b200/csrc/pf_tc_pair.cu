@@ -15,7 +15,7 @@
 //   empty[s]     one per CTA; the leader's tcgen05.commit arrives on both (multicast), releasing the
 //                stage to the producers of both CTAs
 //   acc_full[b]  one per CTA and accumulator buffer, same multicast: buffer b of both CTAs is complete
-//   acc_empty[b] leader's barrier; the four epilogue warps of BOTH CTAs arrive on it once they have
+//   acc_empty[b] leader's barrier; the eight epilogue warps of BOTH CTAs arrive on it once they have
 //                read buffer b out of tensor memory
 // The kernel is persistent: a pair walks over output tiles (pair index, pair index + number of
 // pairs, ...) with two accumulator buffers of 256 columns, so the epilogue of one tile (and the
@@ -35,12 +35,12 @@ namespace pf {
 namespace tc {
 namespace {
 
-constexpr int kPairThreads = 224;   // A producer, MMA issue, 4 epilogue warps, B producer
+constexpr int kPairThreads = 352;   // A producer, MMA issue, 8 epilogue warps, B producer
 constexpr int kPairStages = 6;
 constexpr uint32_t kHalfBytes = 16384;          // 128 rows x 64 bf16
 constexpr uint32_t kPairStageBytes = 2 * kHalfBytes;
 constexpr uint32_t kPairCols = 256;             // fp32 accumulator columns per CTA and buffer
-constexpr uint32_t kPairStaging = 16384;        // 4 epilogue warps x 4 KB store panels
+constexpr uint32_t kPairStaging = 32768;        // 8 epilogue warps x 4 KB store panels
 
 struct PairCtl {
     uint64_t full[kPairStages];
@@ -166,7 +166,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
-            mbar_init(smem_u32(&ctl->acc_empty[b]), 8);   // four epilogue warps of each CTA
+            mbar_init(smem_u32(&ctl->acc_empty[b]), 16);  // eight epilogue warps of each CTA
         }
         ctl->abort = 0;
         fence_barrier_init();
@@ -183,9 +183,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     pdl_launch_dependents();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (warp == 0 || warp == 6) {
+    if (warp == 0 || warp == 10) {
         if (elect_one()) {
-            // ------------------------------------------------------------ producers (A: warp 0, B: warp 6)
+            // ------------------------------------------------------------ producers (A: warp 0, B: warp 10)
             const bool do_a = warp == 0;
             const uint32_t full_leader0 = map_to_cta(smem_u32(&ctl->full[0]), 0);
             uint32_t s = 0, ph = 0;
@@ -257,9 +257,12 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (ok) tc_commit_pair(smem_u32(&ctl->acc_full[buf]));
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 10) {
         // ---------------------------------------------------------------- epilogue (both CTAs, own rows)
+        // eight warps: two per TMEM lane quadrant, each draining two of the four 64-column chunks (with
+        // a short contraction the epilogue of a tile takes as long as its MMAs)
         const int q = warp & 3;
+        const int c_beg = ((warp - 2) >> 2) * 2;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
         // 32 rows x 64 columns staged per warp (128 bytes per row, 16-byte pieces XOR-swizzled by
@@ -277,12 +280,12 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (!mbar_wait_warp(smem_u32(&ctl->acc_full[buf]), (j >> 1) & 1u, abort_flag, p.status)) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < static_cast<int>(kPairCols) / 64; ++c) {
+            for (int c = c_beg; c < c_beg + 2; ++c) {
                 uint32_t v0[32], v1[32];
                 tmem_ld32(lane_base + buf * kPairCols + c * 64, v0);
                 tmem_ld32(lane_base + buf * kPairCols + c * 64 + 32, v1);
                 tmem_ld_wait();
-                if (c == static_cast<int>(kPairCols) / 64 - 1) {
+                if (c == c_beg + 1) {
                     // this warp has read its part of the buffer: hand it back to the leader's MMA thread
                     tc_fence_before();
                     __syncwarp();
