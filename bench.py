@@ -243,6 +243,15 @@ class FfnWorkload:
         self.flat_host.copy_(s["flat"], non_blocking=True)
 
 
+def max_over_ranks(torch, values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (the values themselves when not
+    distributed): a multi-GPU time is the slowest rank's."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
 def time_region(torch, fn, steps, barrier):
     barrier()
     torch.cuda.synchronize()
@@ -338,10 +347,7 @@ def run_ours(args):
     if status != 0:
         raise SystemExit(f"device status {pf.pf_status_string(status)}")
 
-    t = torch.tensor([secs, e2e_secs], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    secs, e2e_secs = float(t[0]), float(t[1])
+    secs, e2e_secs = max_over_ranks(torch, [secs, e2e_secs], dist, device)
     per_step = secs / args.steps
     value = world * w.flops / per_step / 1e12
     byts = sum(sum(linear_bytes(c)) for c in w.cases) + 2 * w.d2h
