@@ -383,7 +383,7 @@ def run_ours(args):
         out["cpu_baseline"] = cpu_baseline(w.cases, w.host)
     if rank == 0:
         if args.suite:
-            from paper_2103_03936_b200 import suite
+            import bench_suite as suite
             del w
             torch.cuda.empty_cache()
             suite.run(args.suite, pk, only=args.suite_only)

@@ -14,7 +14,7 @@ import math
 import torch
 
 import pf_workloads as wl
-from . import binding as pf
+import paper_2103_03936_b200 as pf
 
 L2_BYTES = 126 << 20
 

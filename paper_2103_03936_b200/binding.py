@@ -121,10 +121,17 @@ class _Prepared:
             raise PfError(st, self.where)
 
 
-def _workspace(nbytes: int, device, workspace):
+def _workspace(nbytes: int, device, workspace, stream=None):
+    """The caller's workspace, or a fresh one.  A fresh one is handed back to torch's caching
+    allocator as soon as the wrapper returns, while the kernels that use it may still be queued:
+    that is safe on torch's current stream (the allocator reuses the block in stream order) and is
+    made safe on any other stream by recording that stream on the block."""
     if workspace is not None:
         return workspace
-    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    if stream is not None and stream != torch.cuda.current_stream(device):
+        ws.record_stream(stream)
+    return ws
 
 
 def pf_lowrank_linear_workspace(m, k, n, r, dtype, is_bwd) -> int:
@@ -145,7 +152,7 @@ def pf_lowrank_linear_fwd(x, U, V, *, y=None, T_stash=None, want_stash=False, wo
         y = torch.empty((m, n), dtype=x.dtype, device=x.device)
     if T_stash is None and want_stash:
         T_stash = torch.empty((m, r), dtype=x.dtype, device=x.device)
-    ws = _workspace(pf_lowrank_linear_workspace(m, k, n, r, dt, 0), x.device, workspace)
+    ws = _workspace(pf_lowrank_linear_workspace(m, k, n, r, dt, 0), x.device, workspace, stream)
     args = (_ptr(x), _mat(x, "x"), _ptr(U), _mat(U, "U"), _ptr(V), _mat(V, "V"), _ptr(y), _mat(y, "y"),
             _ptr(T_stash), _mat(T_stash, "T_stash") if T_stash is not None else 0,
             m, k, n, r, dt, _ptr(ws), ws.numel(), _stream(stream))
@@ -190,7 +197,7 @@ def pf_lowrank_linear_bwd(x, U, V, dY, *, T_stash=None, need_dX=True, dX=None, d
         dU = torch.empty((k, r), dtype=x.dtype, device=x.device)
     if dV is None:
         dV = torch.empty((n, r), dtype=x.dtype, device=x.device)
-    ws = _workspace(pf_lowrank_linear_workspace(m, k, n, r, dt, 1), x.device, workspace)
+    ws = _workspace(pf_lowrank_linear_workspace(m, k, n, r, dt, 1), x.device, workspace, stream)
     args = (_ptr(x), _mat(x, "x"), _ptr(U), _mat(U, "U"), _ptr(V), _mat(V, "V"), _ptr(dY), _mat(dY, "dY"),
             _ptr(T_stash), _mat(T_stash, "T_stash") if T_stash is not None else 0,
             _ptr(dX), _mat(dX, "dX") if dX is not None else 0, _ptr(dU), _mat(dU, "dU"),
@@ -231,7 +238,7 @@ def pf_lowrank_conv_fwd(x, U, V, *, stride=1, pad=1, y=None, T_stash=None, want_
     if T_stash is None and want_stash:
         T_stash = torch.empty((N, Ho, Wo, R), dtype=x.dtype, device=x.device)
     ws = _workspace(pf_lowrank_conv_workspace(N, H, W, C, R, O, kh, kw, stride, pad, dt, 0),
-                    x.device, workspace)
+                    x.device, workspace, stream)
     args = (_ptr(x), _ptr(U), _ptr(V), _ptr(y), _ptr(T_stash), N, H, W, C, R, O, kh, kw, stride, pad,
             dt, _ptr(ws), ws.numel(), _stream(stream))
     out = (y, T_stash) if T_stash is not None else y
@@ -255,7 +262,7 @@ def pf_lowrank_conv_bwd(x, U, V, dY, *, stride=1, pad=1, T_stash=None, need_dX=T
     if dV is None:
         dV = torch.empty_like(V)
     ws = _workspace(pf_lowrank_conv_workspace(N, H, W, C, R, O, kh, kw, stride, pad, dt, 1),
-                    x.device, workspace)
+                    x.device, workspace, stream)
     args = (_ptr(x), _ptr(U), _ptr(V), _ptr(dY), _ptr(T_stash), _ptr(dX), _ptr(dU), _ptr(dV),
             N, H, W, C, R, O, kh, kw, stride, pad, dt, _ptr(ws), ws.numel(), _stream(stream))
     if prepare:

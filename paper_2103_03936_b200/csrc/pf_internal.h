@@ -11,7 +11,20 @@
 
 namespace pf {
 
-constexpr int kNumSMs = 148;  // B200
+// Streaming multiprocessors of the current device (148 on B200), asked once per device: grids that
+// must be resident at once (split reductions whose thread blocks meet at counters) and persistent
+// schedules are sized by it.
+inline int num_sms() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }

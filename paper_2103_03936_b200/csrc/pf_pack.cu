@@ -53,6 +53,11 @@ pack_kernel(const PackBatch pb, unsigned char* __restrict__ flat) {
     }
     const int t = lo;
     const int local_chunk = chunk - pb.chunk_prefix[t];
+    // Launched with programmatic stream serialization: the table search above (kernel parameters
+    // only) overlaps the tail of the kernel that produces the gradients; nothing in global memory
+    // is touched before that kernel has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const unsigned char* src = pb.src[t];
     const int64_t bytes = pb.bytes[t];
     unsigned char* dst = flat + pb.dst_byte[t];
@@ -131,9 +136,16 @@ cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const i
             ++i;
         }
         if (pb.count == 0) continue;
-        pack_kernel<<<pb.chunk_prefix[pb.count], kPackThreads, 0, stream>>>(
-            pb, static_cast<unsigned char*>(flat));
-        cudaError_t e = cudaGetLastError();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(pb.chunk_prefix[pb.count]));
+        cfg.blockDim = dim3(kPackThreads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, pack_kernel, pb, static_cast<unsigned char*>(flat));
         if (e != cudaSuccess) return e;
         count_launch();
     }

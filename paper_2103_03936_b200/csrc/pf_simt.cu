@@ -168,8 +168,8 @@ cudaError_t launch_typed(const SimtGemm& g, cudaStream_t stream) {
     count_launch();
     if (g.splits > 1) {
         const int64_t total = g.M * g.N;
-        const int blocks = static_cast<int>(ceil_div(total, 256) < 4 * kNumSMs ? ceil_div(total, 256)
-                                                                                : 4 * kNumSMs);
+        const int blocks = static_cast<int>(ceil_div(total, 256) < 4 * num_sms() ? ceil_div(total, 256)
+                                                                                : 4 * num_sms());
         splitk_reduce_kernel<T><<<blocks, 256, 0, stream>>>(g.partial, g.C, g.ldc, g.M, g.N, g.splits);
         e = cudaGetLastError();
         if (e == cudaSuccess) count_launch();
@@ -230,7 +230,7 @@ repack_multi_kernel(const RepackBatchArgs a) {
 
 int simt_pick_splits(int64_t M, int64_t N, int64_t K) {
     const int64_t tiles = ceil_div(M, BM) * ceil_div(N, BN);
-    int64_t s = ceil_div(2 * kNumSMs, tiles);
+    int64_t s = ceil_div(2 * num_sms(), tiles);
     const int64_t max_by_k = ceil_div(K, 8 * BK);
     if (s > max_by_k) s = max_by_k;
     if (s > 64) s = 64;
@@ -242,7 +242,7 @@ cudaError_t splitk_reduce(const float* partial, void* C, int64_t ldc, int64_t M,
                           int dtype, cudaStream_t stream) {
     const int64_t total = M * N;
     if (total <= 0) return cudaSuccess;
-    const int blocks = static_cast<int>(ceil_div(total, 256) < 4 * kNumSMs ? ceil_div(total, 256) : 4 * kNumSMs);
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 4 * num_sms() ? ceil_div(total, 256) : 4 * num_sms());
     if (dtype == PF_BF16) splitk_reduce_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(partial, C, ldc, M, N, splits);
     else splitk_reduce_kernel<float><<<blocks, 256, 0, stream>>>(partial, C, ldc, M, N, splits);
     cudaError_t e = cudaGetLastError();
@@ -260,8 +260,8 @@ cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t
                              int64_t rows, int64_t cols, int64_t cols_padded, cudaStream_t stream) {
     const int64_t total = rows * cols_padded;
     if (total <= 0) return cudaSuccess;
-    const int blocks = static_cast<int>(ceil_div(total, 256) < 8 * kNumSMs ? ceil_div(total, 256)
-                                                                            : 8 * kNumSMs);
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 8 * num_sms() ? ceil_div(total, 256)
+                                                                            : 8 * num_sms());
     repack_rows_kernel<<<blocks, 256, 0, stream>>>(static_cast<const unsigned short*>(src), ld_src,
                                                    static_cast<unsigned short*>(dst), ld_dst, rows, cols,
                                                    cols_padded);
@@ -299,7 +299,7 @@ cudaError_t repack_rows_bf16_multi(const RepackJob* jobs, int count, cudaStream_
                 a.src[k] = a.src[0]; a.dst[k] = a.dst[0]; a.ld_src[k] = 0; a.ld_dst[k] = 0; a.cols[k] = 0;
                 a.pieces_per_row[k] = 1; a.item_end[k] = total;
             }
-            const long long blocks = ceil_div(total, 256) < 8 * kNumSMs ? ceil_div(total, 256) : 8 * kNumSMs;
+            const long long blocks = ceil_div(total, 256) < 8 * num_sms() ? ceil_div(total, 256) : 8 * num_sms();
             repack_multi_kernel<<<static_cast<int>(blocks), 256, 0, stream>>>(a);
             count_launch();
             cudaError_t e = cudaGetLastError();

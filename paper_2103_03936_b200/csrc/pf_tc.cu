@@ -506,7 +506,7 @@ size_t gemm_smem(int bn, int stages) {
 // one CTA overlap the main loop of the other.
 int pick_stages(int bn, int64_t ctas) {
     const size_t stage = static_cast<size_t>(kBM * kBK * 2 + bn * kBK * 2);
-    const size_t room = (ctas > kNumSMs && bn <= 128) ? (113 * 1024 - 2048) : (200 * 1024 - 2048);
+    const size_t room = (ctas > num_sms() && bn <= 128) ? (113 * 1024 - 2048) : (200 * 1024 - 2048);
     int ns = static_cast<int>(room / stage);
     if (ns > kMaxStages) ns = kMaxStages;
     if (ns < 2) ns = 2;
@@ -557,7 +557,7 @@ int pick_splits(int64_t M, int64_t N, int bn, int64_t K) {
     const int64_t tiles = ceil_div(M, kBM) * ceil_div(N, bn);
     const int64_t nkb = ceil_div(K, kBK);
     if (tiles < 1 || nkb < 1) return 1;
-    int64_t s = kNumSMs / tiles;
+    int64_t s = num_sms() / tiles;
     if (s > nkb / 4) s = nkb / 4;     // at least 4 k-blocks per slice
     if (s > 64) s = 64;
     if (s < 1) s = 1;
@@ -570,7 +570,7 @@ int pick_bn(int64_t N) { return N <= 64 ? 64 : 128; }
 // off as many small single-CTA tiles.
 bool pair_worthwhile(int64_t M, int64_t N, int64_t K) {
     const int64_t tiles = ceil_div(M, 256) * ceil_div(N, 256);
-    return N >= 256 && (tiles >= kNumSMs || (tiles >= 48 && K >= 2048));
+    return N >= 256 && (tiles >= num_sms() || (tiles >= 48 && K >= 2048));
 }
 
 // Slice counts for two products that share one launch (dU: Mu x N, dV: Mv x N, both contracting
@@ -581,10 +581,10 @@ void pick_pair_splits(int64_t Mu, int64_t Mv, int64_t N, int64_t K, int kblock, 
     const int64_t tu = ceil_div(Mu, kBM) * ceil_div(N, bn), tv = ceil_div(Mv, kBM) * ceil_div(N, bn);
     const int64_t nkb = ceil_div(K, kblock);
     *su = 1; *sv = 1;
-    if (tu < 1 || tv < 1 || nkb < 1 || tu + tv > kNumSMs) return;
+    if (tu < 1 || tv < 1 || nkb < 1 || tu + tv > num_sms()) return;
     int64_t best = nkb + 1;
-    for (int64_t a = 1; a <= 64 && a <= nkb && tu * a + tv <= kNumSMs; ++a) {
-        int64_t b = (kNumSMs - tu * a) / tv;
+    for (int64_t a = 1; a <= 64 && a <= nkb && tu * a + tv <= num_sms(); ++a) {
+        int64_t b = (num_sms() - tu * a) / tv;
         if (b > 64) b = 64;
         if (b > nkb) b = nkb;
         if (b < 1) continue;
@@ -613,7 +613,7 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
     // wide outputs that would need more than one wave of 128-column tiles (two CTAs per SM) take
     // 256-column tiles
-    const int bn = (splits <= 1 && N >= 512 && ceil_div(M, kBM) * ceil_div(N, 128) > 2 * kNumSMs) ? 256 : pick_bn(N);
+    const int bn = (splits <= 1 && N >= 512 && ceil_div(M, kBM) * ceil_div(N, 128) > 2 * num_sms()) ? 256 : pick_bn(N);
     CUtensorMap& ta = out->ta;
     CUtensorMap& tb = out->tb;
     bool oka, okb;
@@ -656,7 +656,7 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     p.counters = nullptr;
     if (p.splits > 1) {
         // the CTAs of a tile wait for one another, so all of them must be resident at once
-        if (static_cast<int64_t>(grid.x) * grid.y > kFixTiles || static_cast<int64_t>(grid.x) * grid.y * grid.z > kNumSMs ||
+        if (static_cast<int64_t>(grid.x) * grid.y > kFixTiles || static_cast<int64_t>(grid.x) * grid.y * grid.z > num_sms() ||
             bn == 256 || partial == nullptr)
             return PF_ERR_UNSUPPORTED;
         // the slices of a CTA's share are gathered in the pipeline stages
@@ -669,6 +669,14 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     out->grid = grid;
     out->bn = bn;
     return PF_OK;
+}
+
+// Launches one prepared product on its own.
+int launch_prepared(const GemmLaunch& g, cudaStream_t stream) {
+    const cudaError_t e = g.bn == 64    ? launch_gemm<64>(g.ta, g.tb, g.p, g.grid, stream)
+                          : g.bn == 128 ? launch_gemm<128>(g.ta, g.tb, g.p, g.grid, stream)
+                                        : launch_gemm<256>(g.ta, g.tb, g.p, g.grid, stream);
+    return e == cudaSuccess ? PF_OK : PF_ERR_CUDA;
 }
 
 // `copy2` (optional): asks for a second copy of C at pitch ldc2; *copy2_done tells whether the launch
@@ -718,7 +726,7 @@ int gemm_multi(const GemmLaunch* const* g, int count, cudaStream_t stream) {
             seen_plain = true;
         }
     }
-    if (split_ctas > kNumSMs) return PF_ERR_UNSUPPORTED;
+    if (split_ctas > num_sms()) return PF_ERR_UNSUPPORTED;
     GemmParams prm[3];
     size_t smem = 0;
     for (int i = 0; i < 3; ++i) {
@@ -818,6 +826,8 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
 int linear_fwd(const LinearArgs& a, int* handled) {
     *handled = 0;
     if (encode_fn() == nullptr) return PF_OK;
+    // the grids below index column tiles with 16 bits: absurdly wide layers take the FMA kernels
+    if (a.k > (1 << 22) || a.n > (1 << 22) || a.r > (1 << 22)) return PF_OK;
     int st = PF_OK;
     char* scratch = a.ws;
     Staged x, U, V;
@@ -857,6 +867,8 @@ int linear_fwd(const LinearArgs& a, int* handled) {
 int linear_bwd(const LinearArgs& a, int* handled) {
     *handled = 0;
     if (encode_fn() == nullptr) return PF_OK;
+    // the grids below index column tiles with 16 bits: absurdly wide layers take the FMA kernels
+    if (a.k > (1 << 22) || a.n > (1 << 22) || a.r > (1 << 22)) return PF_OK;
     int st = PF_OK;
     char* scratch = a.ws;
     Staged x, U, V, dY, T;
@@ -992,52 +1004,57 @@ int conv_bwd(const ConvArgs& a, int* handled) {
     const int64_t M = static_cast<int64_t>(a.N) * a.H * a.W, Keff = static_cast<int64_t>(a.kh) * a.kw * a.C;
     ChainPlan plan;
     if (!a.T && !chain_plan(M, Keff, a.O, a.R, false, &plan)) return PF_OK;
-    *handled = 1;
     int st;
-    const void* T = a.T;
-    if (!T) {   // recompute the thin convolution (phase 1 of the forward only)
-        const ChainConv cv{a.N, a.H, a.W, a.C, a.kh, a.kw, a.pad};
-        st = chain(a.x, a.C, M, Keff, a.U, a.R, a.R, a.V, a.R, a.O, nullptr, a.O, a.ws_T, a.R, a.stream, &cv);
-        if (st != PF_OK) return st;
-        T = a.ws_T;
-    }
+    const void* T = a.T ? a.T : a.ws_T;
     void* dT = a.ws_G;
     int su, sv;
     pick_pair_splits(Keff, a.O, a.R, M, conv_box_h(a.H, a.W, 64) * a.W, &su, &sv);
     float* pu = reinterpret_cast<float*>(a.ws);
     float* pv = reinterpret_cast<float*>(a.ws + align_up(partial_bytes(Keff, a.R, su), 256));
-    // dT = dY V  (per pixel)
-    st = gemm({a.dY, a.O, false}, {a.V, a.R, true}, M, a.R, a.O, dT, a.R, 1, nullptr, a.stream);
-    if (st != PF_OK) return st;
+    // Every product is prepared (tensor maps, geometry; nothing launched) before the call is
+    // accepted, so a shape that one of them cannot take still reaches the FMA kernels.
     // dU[tap] = shifted x^T dT ; dV = dY^T T   (reductions over all pixels, split across CTAs)
     // dX = sum over taps of shifted dT times U[tap]^T  (implicit GEMM, contraction kh*kw*R)
-    // All three depend on dT only and share one launch: the few long CTAs of the split reductions
-    // start first and the many short dX tiles fill the second CTA slot of every SM beside them.
     const ConvA cu{2, a.N, a.H, a.W, a.C, a.kw, a.pad, a.C};
     const ConvA cx{1, a.N, a.H, a.W, a.R, a.kw, a.pad, a.C};
-    GemmLaunch gu, gv, gx;
-    st = gemm_prepare({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, &cu, &gu);
+    GemmLaunch gt, gu, gv, gx;
+    auto prepare = [](const Operand& A, const Operand& B, int64_t Mm, int64_t Nn, int64_t Kk, void* C, int64_t ldc,
+                      int splits, float* partial, const ConvA* cv, GemmLaunch* out) {
+        int r = gemm_prepare(A, B, Mm, Nn, Kk, C, ldc, splits, partial, cv, out);
+        if (r == PF_ERR_UNSUPPORTED && splits > 1) r = gemm_prepare(A, B, Mm, Nn, Kk, C, ldc, 1, nullptr, cv, out);
+        return r;
+    };
+    st = prepare({a.dY, a.O, false}, {a.V, a.R, true}, M, a.R, a.O, dT, a.R, 1, nullptr, nullptr, &gt);
+    if (st == PF_OK) st = prepare({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, &cu, &gu);
+    if (st == PF_OK) st = prepare({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, nullptr, &gv);
+    if (st == PF_OK && a.dX)
+        st = prepare({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
+                     nullptr, &cx, &gx);
+    if (st == PF_ERR_UNSUPPORTED) return PF_OK;      // declined: nothing has been launched
     if (st != PF_OK) return st;
-    st = gemm_prepare({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, nullptr, &gv);
-    if (st != PF_OK) return st;
-    if (a.dX) {
-        st = gemm_prepare({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
-                          nullptr, &cx, &gx);
+    *handled = 1;
+    if (!a.T) {   // recompute the thin convolution (phase 1 of the forward only)
+        const ChainConv cv{a.N, a.H, a.W, a.C, a.kh, a.kw, a.pad};
+        st = chain(a.x, a.C, M, Keff, a.U, a.R, a.R, a.V, a.R, a.O, nullptr, a.O, a.ws_T, a.R, a.stream, &cv);
         if (st != PF_OK) return st;
     }
+    // dT = dY V  (per pixel)
+    st = launch_prepared(gt, a.stream);
+    if (st != PF_OK) return st;
+    // dU, dV and dX depend on dT only and share one launch: the few long CTAs of the split reductions
+    // start first and the many short dX tiles fill the second CTA slot of every SM beside them.
     const GemmLaunch* list[3] = {&gu, &gv, &gx};
     if (gu.p.splits <= 1 && gv.p.splits > 1) { list[0] = &gv; list[1] = &gu; }
     st = gemm_multi(list, a.dX ? 3 : 2, a.stream);
     if (st != PF_ERR_UNSUPPORTED) return st;
     // separate launches (tile widths that cannot share one)
     if (a.dX) {
-        st = gemm({dT, a.R, false}, {a.U, a.R, false}, M, a.C, static_cast<int64_t>(a.kh) * a.kw * a.R, a.dX, a.C, 1,
-                  nullptr, a.stream, &cx);
+        st = launch_prepared(gx, a.stream);
         if (st != PF_OK) return st;
     }
-    st = gemm({a.x, a.C, true}, {dT, a.R, true}, Keff, a.R, M, a.dU, a.R, su, pu, a.stream, &cu);
+    st = launch_prepared(gu, a.stream);
     if (st != PF_OK) return st;
-    return gemm({a.dY, a.O, true}, {T, a.R, true}, a.O, a.R, M, a.dV, a.R, sv, pv, a.stream);
+    return launch_prepared(gv, a.stream);
 }
 
 }  // namespace tc

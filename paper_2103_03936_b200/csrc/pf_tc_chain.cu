@@ -379,8 +379,8 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
     int64_t best = 1;
     if (has_out) {
         double best_cost = 1e30;
-        for (int64_t s = 1; s <= nt && (s == 1 || row_tiles * s <= kNumSMs); ++s) {
-            const double waves = static_cast<double>(ceil_div(row_tiles * s, kNumSMs));
+        for (int64_t s = 1; s <= nt && (s == 1 || row_tiles * s <= num_sms()); ++s) {
+            const double waves = static_cast<double>(ceil_div(row_tiles * s, num_sms()));
             const double cost = waves * (static_cast<double>(K1) + 128.0 * ceil_div(nt, s));
             if (cost < best_cost * 0.97) { best_cost = cost; best = s; }
         }

@@ -350,7 +350,7 @@ int gemm_pair_2sm(const void* A, int64_t lda, bool a_mn, const void* B, int64_t 
     if ((reinterpret_cast<uintptr_t>(C) & 15) != 0 || ldc % 8 != 0) return PF_ERR_UNSUPPORTED;
     const int64_t tiles_m = ceil_div(M, 256), tiles_n = ceil_div(N, 256);
     if (tiles_m * tiles_n > 0x7fffffff) return PF_ERR_UNSUPPORTED;
-    const int64_t pairs = std::min<int64_t>(tiles_m * tiles_n, kNumSMs / 2);   // persistent: one CTA per SM
+    const int64_t pairs = std::min<int64_t>(tiles_m * tiles_n, num_sms() / 2);   // persistent: one CTA per SM
     CUtensorMap ta, tb;
     const bool oka = a_mn ? cached_map_2d(&ta, A, K, M, lda, 64) : cached_map_2d(&ta, A, M, K, lda, 128);
     const bool okb = b_mn ? cached_map_2d(&tb, B, K, N, ldb, 64) : cached_map_2d(&tb, B, N, K, ldb, 128);

@@ -70,12 +70,24 @@ def normal(seed: int, stream: int, shape, sigma: float = 1.0) -> np.ndarray:
 
 
 def round_to(a64: np.ndarray, dtype: str) -> np.ndarray:
-    """Round fp64 values once to the storage type (RNE)."""
-    f32 = np.ascontiguousarray(a64, dtype=np.float32)
+    """Round fp64 values once to the storage type (RNE).
+
+    bf16 is reached in one rounding step: the fp64 value is first narrowed to fp32 with
+    round-to-odd (truncate, then set the last bit when anything was cut off), which keeps
+    enough information for the final round-to-nearest-even to 8 significand bits to be
+    the correctly rounded bf16 of the fp64 value (no double rounding)."""
+    a64 = np.ascontiguousarray(a64, dtype=np.float64)
+    f32 = a64.astype(np.float32)
     if dtype == F32:
         return f32
     if dtype == BF16:
-        bits = f32.view(np.uint32)
+        back = f32.astype(np.float64)
+        inexact = back != a64
+        # truncate toward zero where RNE went away from zero, then force the last bit odd
+        away = inexact & (np.abs(back) > np.abs(a64))
+        bits = f32.view(np.uint32).copy()
+        bits[away] -= np.uint32(1)
+        bits[inexact] |= np.uint32(1)
         bias = np.uint32(0x7FFF) + ((bits >> np.uint32(16)) & np.uint32(1))
         return ((bits + bias) >> np.uint32(16)).astype(np.uint16)
     raise ValueError(dtype)

@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2103_03936_b200 as pf
 import pf_workloads as wl
-from _gpu import Guarded, assert_close, dev
+from _gpu import ESCAPES, Guarded, assert_blocks_close, assert_close, dev
 
 pytestmark = pytest.mark.gpu
 
@@ -32,13 +32,14 @@ def run_conv(case, stash=True, need_dX=True, tiny=False):
         aw = {k_: np.abs(oracle.widen(v)) for k_, v in d.items()}
         ab["y"], ab["T"] = oracle.conv_fwd(aw["x"], aw["U"], aw["V"], case.stride, case.pad)
         ab["dX"], ab["dU"], ab["dV"] = oracle.conv_bwd(aw["x"], aw["U"], aw["V"], aw["dY"], case.stride, case.pad)
-    errs = {"y": assert_close(gy.t, y_ref, dt, "y", abs_ref64=ab.get("y"))}
+    tag = f"{case.name} {case.N}x{case.H}x{case.W} {case.C}->{case.R}->{case.O} k{case.kh} s{case.stride} {dt} "
+    checks = [("y", gy, y_ref)]
     if stash:
-        errs["T"] = assert_close(gT.t, T_ref, dt, "T", abs_ref64=ab.get("T"))
+        checks.append(("T", gT, T_ref))
     if need_dX:
-        errs["dX"] = assert_close(gdX.t, dX_ref, dt, "dX", abs_ref64=ab.get("dX"))
-    errs["dU"] = assert_close(gdU.t, dU_ref, dt, "dU", abs_ref64=ab.get("dU"))
-    errs["dV"] = assert_close(gdV.t, dV_ref, dt, "dV", abs_ref64=ab.get("dV"))
+        checks.append(("dX", gdX, dX_ref))
+    checks += [("dU", gdU, dU_ref), ("dV", gdV, dV_ref)]
+    errs = {nm: assert_close(g.t, ref, dt, tag + nm, abs_ref64=ab.get(nm)) for nm, g, ref in checks}
     for g in (gy, gT, gdX, gdU, gdV):
         g.check()
     assert pf.pf_last_device_status() == 0
@@ -58,10 +59,20 @@ SMALL = [  # N,H,W,C,R,O,k,stride,pad
 ]
 
 
+# bf16 outputs of the small shapes that may be judged against the magnitude of their summands
+# (single near-cancelled sums, see _gpu.assert_close); fixed by the seeded inputs.
+MAX_CANCELLED_OUTPUTS = 1
+
+
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_small_shapes(dtype):
+    first = len(ESCAPES)
     for i, (N, H, W, C, R, O, k, st, pad) in enumerate(SMALL):
         run_conv(wl.ConvCase(f"s{i}", N, H, W, C, R, O, dtype, 50 + i, kh=k, kw=k, stride=st, pad=pad), tiny=True)
+    took = ESCAPES[first:]
+    for what, rel, ratio, err_abs in took:
+        print(f"cancelled output {what}: rel {rel:.2e}, |exact|/|summands| {ratio:.2e}, err vs summands {err_abs:.2e}")
+    assert len(took) <= (MAX_CANCELLED_OUTPUTS if dtype == wl.BF16 else 0), took
 
 
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
@@ -76,10 +87,14 @@ def test_multi_tile(dtype, N, H, W, C, R, O):
                                            (2, 32, 32, 128, 128, 256, 5), (2, 8, 16, 128, 192, 64, 1),
                                            (3, 14, 14, 128, 64, 128, 3), (2, 7, 7, 256, 64, 64, 3),
                                            (2, 28, 28, 128, 64, 72, 3), (3, 10, 6, 128, 64, 64, 3),
-                                           (1, 3, 64, 128, 64, 64, 3)])
+                                           (1, 3, 64, 128, 64, 64, 3),
+                                           (2, 16, 16, 128, 256, 64, 3), (2, 16, 16, 128, 320, 128, 3),
+                                           (2, 16, 16, 128, 384, 72, 3)])
 def test_tensor_core_envelope(N, H, W, C, R, O, k):
     """Shapes inside the implicit-GEMM tensor-core envelope (stride 1, 'same' padding, C % 128 == 0,
-    R % 64 == 0, image rows packing into 128- and 64-pixel tiles), with and without stash / dX."""
+    R % 64 == 0, image rows packing into 128- and 64-pixel tiles), with and without stash / dX.  The
+    ranks 256, 320 and 384 reach the parts of the fused kernel that only ranks above 192 use (a
+    second group of first-product MMAs, the short ring, store staging inside the ring stages)."""
     run_conv(wl.ConvCase("tc", N, H, W, C, R, O, wl.BF16, 63, kh=k, kw=k, pad=(k - 1) // 2))
     run_conv(wl.ConvCase("tc", N, H, W, C, R, O, wl.BF16, 64, kh=k, kw=k, pad=(k - 1) // 2), stash=False,
              need_dX=False)
@@ -102,13 +117,14 @@ def test_configs_full_size_sampled(name, imgs):
     torch.cuda.synchronize()
     y_ref, T_ref = oracle.conv_fwd(d["x"][imgs], d["U"], d["V"])
     dX_ref, _, _ = oracle.conv_bwd(d["x"][imgs], d["U"], d["V"], d["dY"][imgs])
-    assert_close(y[imgs], y_ref, c.dtype, "y")
-    assert_close(T[imgs], T_ref, c.dtype, "T")
-    assert_close(dX[imgs], dX_ref, c.dtype, "dX")
+    for got, want, nm in ((y[imgs], y_ref, "y"), (T[imgs], T_ref, "T"), (dX[imgs], dX_ref, "dX")):
+        assert_close(got, want, c.dtype, nm)
+        assert_blocks_close(got, want, c.dtype, nm)          # 128 pixels x 128 channels per block
     J = [0, 31, 63]
     _, dU_ref, dV_ref = oracle.conv_bwd(d["x"], d["U"][..., J], d["V"][:, J], d["dY"])
-    assert_close(dU[..., J], dU_ref, c.dtype, "dU")
-    assert_close(dV[:, J], dV_ref, c.dtype, "dV")
+    for got, want, nm in ((dU[..., J], dU_ref, "dU"), (dV[:, J], dV_ref, "dV")):
+        assert_close(got, want, c.dtype, nm)
+        assert_blocks_close(got, want, c.dtype, nm)          # 128 rows x the sampled columns per block
     # the step ends with the flat gradient buffer of its factor gradients
     flat, offs = pf.pf_pack_factor_grads([dU, dV])
     torch.cuda.synchronize()

@@ -8,12 +8,12 @@ import torch
 import oracle
 import paper_2103_03936_b200 as pf
 import pf_workloads as wl
-from _gpu import Guarded, assert_close, dev, host
+from _gpu import ESCAPES, Guarded, assert_blocks_close, assert_close, dev, host
 
 pytestmark = pytest.mark.gpu
 
 
-def run_case(case, ld_pad=0, stash=True, need_dX=True, tiny=False):
+def run_case(case, ld_pad=0, stash=True, need_dX=True, tiny=False, blocks=False):
     d = case.generate()
     dt = case.dtype
     m, k, n, r = case.m, case.k, case.n, case.r
@@ -42,13 +42,18 @@ def run_case(case, ld_pad=0, stash=True, need_dX=True, tiny=False):
         aw = {k_: np.abs(oracle.widen(v)) for k_, v in d.items()}
         ab["y"], ab["T"] = oracle.linear_fwd(aw["x"], aw["U"], aw["V"])
         ab["dX"], ab["dU"], ab["dV"] = oracle.linear_bwd(aw["x"], aw["U"], aw["V"], aw["dY"])
-    errs = {"y": assert_close(gy.t, y_ref, dt, "y", abs_ref64=ab.get("y"))}
+    tag = f"{case.name} {m}x{k}->{n} r{r} {dt} "
+    checks = [("y", gy, y_ref)]
     if stash:
-        errs["T"] = assert_close(gT.t, T_ref, dt, "T", abs_ref64=ab.get("T"))
+        checks.append(("T", gT, T_ref))
     if need_dX:
-        errs["dX"] = assert_close(gdX.t, dX_ref, dt, "dX", abs_ref64=ab.get("dX"))
-    errs["dU"] = assert_close(gdU.t, dU_ref, dt, "dU", abs_ref64=ab.get("dU"))
-    errs["dV"] = assert_close(gdV.t, dV_ref, dt, "dV", abs_ref64=ab.get("dV"))
+        checks.append(("dX", gdX, dX_ref))
+    checks += [("dU", gdU, dU_ref), ("dV", gdV, dV_ref)]
+    errs = {}
+    for nm, g, ref in checks:
+        errs[nm] = assert_close(g.t, ref, dt, tag + nm, abs_ref64=ab.get(nm))
+        if blocks:   # and no 128 x 128 block of the tensor may miss the same bound
+            errs[nm + " worst block"] = assert_blocks_close(g.t, ref, dt, tag + nm)
     for g in (gy, gT, gdX, gdU, gdV):
         g.check()
     assert pf.pf_last_device_status() == 0
@@ -58,10 +63,20 @@ def run_case(case, ld_pad=0, stash=True, need_dX=True, tiny=False):
 GRID = [(m, k, n, r) for m, k, n, r in itertools.product((1, 7, 130), (1, 17, 100), (3, 24, 130), (1, 5, 33))]
 
 
+# Outputs of the bf16 grid that may be judged against the magnitude of their summands (see
+# _gpu.assert_close): single near-cancelled sums.  The count is fixed by the seeded inputs.
+MAX_CANCELLED_OUTPUTS = 2
+
+
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_tiny_exhaustive_grid(dtype):
+    first = len(ESCAPES)
     for idx, (m, k, n, r) in enumerate(GRID):
         run_case(wl.LinearCase(f"g{idx}", m, k, n, r, dtype, 100 + idx), tiny=True)
+    took = ESCAPES[first:]
+    for what, rel, ratio, err_abs in took:
+        print(f"cancelled output {what}: rel {rel:.2e}, |exact|/|summands| {ratio:.2e}, err vs summands {err_abs:.2e}")
+    assert len(took) <= (MAX_CANCELLED_OUTPUTS if dtype == wl.BF16 else 0), took
 
 
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
@@ -75,8 +90,9 @@ def test_multi_tile_ragged(dtype, m, k, n, r):
                                      (4100, 72, 1000, 130), (2048, 64, 64, 256), (2304, 520, 264, 320),
                                      (2050, 100, 130, 33)])
 def test_fused_chain_envelope(m, k, n, r):
-    """m >= 2048 takes the fused two-GEMM kernel: every rank padding (64..384), ragged row tile,
-    ragged k / n tails, with and without stash and dX."""
+    """m >= 2048 with r <= 192 takes the fused two-GEMM kernel (rank paddings 64, 128, 192; ragged
+    row tile, ragged k / n tails, with and without stash and dX); the larger ranks of this list run
+    as unfused products on the same batch sizes."""
     run_case(wl.LinearCase("chain", m, k, n, r, wl.BF16, 13))
     run_case(wl.LinearCase("chain", m, k, n, r, wl.BF16, 14), stash=False, need_dX=False)
 
@@ -106,7 +122,7 @@ def test_config_C1_tiny_fp32():
 
 @pytest.mark.parametrize("name", ["C2a", "C2b", "C3i", "C3h"])
 def test_configs_full_size(name):
-    errs = run_case(wl.linear_cases()[name])
+    errs = run_case(wl.linear_cases()[name], blocks=True)
     print(name, errs)
 
 
@@ -154,13 +170,14 @@ def test_rank_sweep_full_size_sampled(sweep_inputs, r):
     rows = [0, 1, 127, 128, 5000, 8191, 8192, 16383]
     y_ref, T_ref = oracle.linear_fwd(x_h[rows], U_h, V_h)
     dX_ref, _, _ = oracle.linear_bwd(x_h[rows], U_h, V_h, dY_h[rows])
-    assert_close(y[rows], y_ref, c.dtype, "y rows")
-    assert_close(T[rows], T_ref, c.dtype, "T rows")
-    assert_close(dX[rows], dX_ref, c.dtype, "dX rows")
+    for got, want, nm in ((y[rows], y_ref, "y rows"), (T[rows], T_ref, "T rows"), (dX[rows], dX_ref, "dX rows")):
+        assert_close(got, want, c.dtype, nm)
+        assert_blocks_close(got, want, c.dtype, nm)          # 8 sampled rows x 128 columns per block
     J = sorted({0, r // 2, r - 1})
     _, dU_ref, dV_ref = oracle.linear_bwd(x_h, U_h[:, J], V_h[:, J], dY_h)
-    assert_close(dU[:, J], dU_ref, c.dtype, "dU cols")
-    assert_close(dV[:, J], dV_ref, c.dtype, "dV cols")
+    for got, want, nm in ((dU[:, J], dU_ref, "dU cols"), (dV[:, J], dV_ref, "dV cols")):
+        assert_close(got, want, c.dtype, nm)
+        assert_blocks_close(got, want, c.dtype, nm)          # 128 rows x the sampled columns per block
     assert pf.pf_last_device_status() == 0
 
 

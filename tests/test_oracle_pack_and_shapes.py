@@ -79,6 +79,25 @@ def test_generator_is_deterministic_and_rounded_once():
     # bf16 RNE: 1 + 2^-8 is a tie and rounds to even (1.0); 1 + 3*2^-9 rounds up
     r = wl.round_to(np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -9, -2.5]), wl.BF16)
     np.testing.assert_array_equal(oracle.widen(r), [1.0, 1.0 + 2.0 ** -7, -2.5])
+    # one rounding, not two: just above / below a bf16 tie by less than fp32 can hold (going
+    # through fp32 first would land on the tie and then on the even neighbour)
+    eps = 2.0 ** -40
+    r = wl.round_to(np.array([1.0 + 2.0 ** -8 + eps, 1.0 + 3 * 2.0 ** -8 - eps,
+                              -(1.0 + 2.0 ** -8 + eps), -(1.0 + 3 * 2.0 ** -8 - eps)]), wl.BF16)
+    np.testing.assert_array_equal(oracle.widen(r), [1.0 + 2.0 ** -7, 1.0 + 2.0 ** -7,
+                                                    -(1.0 + 2.0 ** -7), -(1.0 + 2.0 ** -7)])
+    # agreement with an exact rational rounding on random values
+    from fractions import Fraction
+    vals = wl.normal(77, 0, (300,))
+    got = oracle.widen(wl.round_to(vals, wl.BF16))
+    for v, g in zip(vals, got):
+        e = int(np.floor(np.log2(abs(v))))
+        ulp = Fraction(2) ** (e - 7)
+        q = Fraction(v) / ulp
+        lo = q.numerator // q.denominator
+        frac = q - lo
+        n = lo + (1 if frac > Fraction(1, 2) or (frac == Fraction(1, 2) and lo % 2) else 0)
+        assert Fraction(g) == n * ulp
 
 
 def test_generator_distributions():
