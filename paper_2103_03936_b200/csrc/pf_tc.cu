@@ -67,6 +67,7 @@ struct GemmParams {
     int rows_tile;           // output rows per CTA: 128, or cv_box_h * W pixels for conv_mode 1
     int kpix;                // conv_mode 2: pixels per k-block (cv_box_h * W <= 64), else 64
     int nkb_total;           // k-blocks of the whole contraction
+    int independent;         // 1: reads nothing the preceding kernel of the stream writes (see gemm_tile)
 };
 
 __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
@@ -132,7 +133,11 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    pdl_wait();                 // everything above overlapped the previous kernel's tail
+    // A product marked independent reads nothing that the kernel launched just before it writes, so
+    // it does not wait for that kernel: its blocks run beside it on SMs that kernel leaves free.  (Every
+    // kernel of this library lets its successor start only after its own wait has returned, i.e. once
+    // everything older in the stream is complete, so older results are safe to read.)
+    if (!p.independent) pdl_wait();     // everything above overlapped the previous kernel's tail
     pdl_launch_dependents();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -593,6 +598,30 @@ void pick_pair_splits(int64_t Mu, int64_t Mv, int64_t N, int64_t K, int kblock, 
     }
 }
 
+// Slices of dU (k x r) and dV (n x r) in the backward of the linear layer, and whether dV runs BESIDE
+// the fused dX kernel instead of after it.  dV = dY^T T needs nothing that kernel writes.  When the
+// contraction of its first product is long against its output (n >= 2k), the fused kernel is left
+// unsplit (one block per 128-row tile, no block repeats another's first product), which leaves SMs
+// free; the dV blocks are sized to exactly those SMs and do not wait for the fused kernel, and the
+// dU blocks (which need G) follow on the SMs the fused kernel vacates.
+void bwd_split_plan(int64_t m, int64_t k, int64_t n, int64_t r, bool fused_dx, int* su, int* sv, bool* beside) {
+    pick_pair_splits(k, n, r, m, kBK, su, sv);
+    *beside = false;
+    if (!fused_dx || n < 2 * k) return;
+    const int bn = pick_bn(r);
+    const int64_t row_tiles = ceil_div(m, kBM), nkb = ceil_div(m, kBK);
+    const int64_t tu = ceil_div(k, kBM) * ceil_div(r, bn), tv = ceil_div(n, kBM) * ceil_div(r, bn);
+    const int64_t free_sms = num_sms() - row_tiles;
+    const int64_t smax = std::max<int64_t>(1, std::min<int64_t>(64, nkb / 4));
+    if (free_sms < tv || tu + tv > num_sms()) return;
+    const int64_t b = std::min(free_sms / tv, smax);
+    const int64_t a = std::min((num_sms() - tv * b) / tu, smax);
+    if (a < 1 || b < 1) return;
+    *su = static_cast<int>(a);
+    *sv = static_cast<int>(b);
+    *beside = true;
+}
+
 // C[M,N] (bf16, ldc) = A * B.  `partial` must hold splits*M*N floats when splits > 1.
 struct ConvA {
     int mode;                   // 1: dX (A = dT image), 2: dU (A = x image)
@@ -654,6 +683,7 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     p.bn = bn;
     p.num_stages = pick_stages(bn, static_cast<int64_t>(grid.x) * grid.y * grid.z);
     p.counters = nullptr;
+    p.independent = 0;
     if (p.splits > 1) {
         // the CTAs of a tile wait for one another, so all of them must be resident at once
         if (static_cast<int64_t>(grid.x) * grid.y > kFixTiles || static_cast<int64_t>(grid.x) * grid.y * grid.z > num_sms() ||
@@ -813,9 +843,13 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
     if (bwd) {
         b += repack_room(m, n);                                             // dY
         b += align_up(static_cast<size_t>(m) * pad8(r) * 2, 256);           // G at padded pitch
-        int su, sv;
-        pick_pair_splits(k, n, r, m, kBK, &su, &sv);
-        b += align_up(partial_bytes(k, r, su), 256) + align_up(partial_bytes(n, r, sv), 256);
+        // slices for either backward structure (the choice depends on pointers the query does not see)
+        int su, sv, su2, sv2;
+        bool beside;
+        bwd_split_plan(m, k, n, r, false, &su, &sv, &beside);
+        bwd_split_plan(m, k, n, r, true, &su2, &sv2, &beside);
+        b += align_up(std::max(partial_bytes(k, r, su), partial_bytes(k, r, su2)), 256) +
+             align_up(std::max(partial_bytes(n, r, sv), partial_bytes(n, r, sv2)), 256);
     }
     // skinny batches: the m x r products (x U, dY V) are split over their contraction to fill the SMs
     const int s1 = std::max(pick_splits(m, r, pick_bn(r), k), bwd ? pick_splits(m, r, pick_bn(r), n) : 1);
@@ -898,12 +932,27 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     char* G = scratch;
     const int64_t ldG = pad8(a.r);
     scratch += align_up(static_cast<size_t>(a.m) * ldG * 2, 256);
+    size_t pu_bytes = 0, pv_bytes = 0;
+    ChainPlan plan;
+    const bool fused_dx = use_chain(a.m, a.r) && (!a.dX || tma_ok(a.dX, a.lddx)) &&
+                          chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan);
     int su, sv;
-    pick_pair_splits(a.k, a.n, a.r, a.m, kBK, &su, &sv);
+    bool dv_beside;
+    bwd_split_plan(a.m, a.k, a.n, a.r, fused_dx, &su, &sv, &dv_beside);
+    {   // the workspace holds room for the slices of either structure (see linear_extra_workspace)
+        int s0, s1, s2, s3;
+        bool unused;
+        bwd_split_plan(a.m, a.k, a.n, a.r, false, &s0, &s1, &unused);
+        bwd_split_plan(a.m, a.k, a.n, a.r, true, &s2, &s3, &unused);
+        const size_t bu = std::max(partial_bytes(a.k, a.r, s0), partial_bytes(a.k, a.r, s2));
+        const size_t bv = std::max(partial_bytes(a.n, a.r, s1), partial_bytes(a.n, a.r, s3));
+        pu_bytes = align_up(bu, 256);
+        pv_bytes = align_up(bv, 256);
+    }
     float* pu = reinterpret_cast<float*>(scratch);
-    scratch += align_up(partial_bytes(a.k, a.r, su), 256);
+    scratch += pu_bytes;
     float* pv = reinterpret_cast<float*>(scratch);
-    scratch += align_up(partial_bytes(a.n, a.r, sv), 256);
+    scratch += pv_bytes;
     float* p1 = reinterpret_cast<float*>(scratch);
     // G = dY V ; dX = G U^T ; dU = x^T G ; dV = dY^T T
     if (need_T) {   // no stash: recompute T = x U
@@ -911,10 +960,10 @@ int linear_bwd(const LinearArgs& a, int* handled) {
                   pick_splits(a.m, a.r, pick_bn(a.r), a.k), p1, a.stream);
         if (st != PF_OK) return st;
     }
-    ChainPlan plan;
     bool dx_pending = false;     // dX still to be computed as a plain product G U^T
-    if (use_chain(a.m, a.r) && (!a.dX || tma_ok(a.dX, a.lddx)) && chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan)) {
-        st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream);
+    if (fused_dx) {
+        st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream, nullptr,
+                   dv_beside ? 1 : 0);
         if (st != PF_OK) return st;
     } else {
         st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG,
@@ -932,6 +981,12 @@ int linear_bwd(const LinearArgs& a, int* handled) {
             const GemmLaunch* list[3] = {&gu, &gv, &gx};
             // a split product has to come before the plain ones
             if (gu.p.splits <= 1 && gv.p.splits > 1) { list[0] = &gv; list[1] = &gu; }
+            if (dv_beside && !dx_pending) {
+                // dV first (its blocks are dispatched first, onto the SMs the fused kernel left free) and
+                // without waiting for the fused kernel; dU follows as that kernel's blocks retire
+                gv.p.independent = 1;
+                list[0] = &gv; list[1] = &gu;
+            }
             st = gemm_multi(list, dx_pending ? 3 : 2, a.stream);
             if (st != PF_ERR_UNSUPPORTED) return st;
             if (dx_pending) {

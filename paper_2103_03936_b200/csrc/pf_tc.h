@@ -34,7 +34,9 @@ struct ChainPlan {
     int r_pad, num_stages, stage_bytes, nsplit, tiles_per_split, row_tiles, boxes_per_stage, staging_off;
     size_t smem;
 };
-bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan, int rows_tile = 128);
+// `max_split` caps the number of column ranges the output is split into (0 = no cap).
+bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan, int rows_tile = 128,
+                int max_split = 0);
 int conv_box_h(int H, int W, int limit);
 // When `conv` is given, A is an NHWC image and phase 1 is the implicit GEMM of a kh x kw, stride-1,
 // "same"-padded convolution: M = N*H*W pixels, K1 = kh*kw*C, B1 = U as a (kh*kw*C) x r matrix.
@@ -43,7 +45,7 @@ struct ChainConv {
 };
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
-          cudaStream_t stream, const ChainConv* conv = nullptr);
+          cudaStream_t stream, const ChainConv* conv = nullptr, int max_split = 0);
 
 // Plain product on CTA pairs (pf_tc_pair.cu); PF_ERR_UNSUPPORTED when the output is not 16-byte aligned
 // with a pitch that is a multiple of 8 elements.

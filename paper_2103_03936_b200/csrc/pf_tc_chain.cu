@@ -362,7 +362,7 @@ int conv_box_h(int H, int W, int limit) {
 }
 
 // Shape envelope of the fused kernel and its launch geometry.
-bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan, int rows_tile) {
+bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, ChainPlan* plan, int rows_tile, int max_split) {
     const int64_t r_pad = (r + 63) / 64 * 64;
     if (r_pad > 384 || M > 0x7fffffff || K1 > 0x7fffffff || N2 > 0x7fffffff) return false;
     const int64_t stage = kTileBytes + r_pad * 128;
@@ -379,7 +379,7 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
     int64_t best = 1;
     if (has_out) {
         double best_cost = 1e30;
-        for (int64_t s = 1; s <= nt && (s == 1 || row_tiles * s <= num_sms()); ++s) {
+        for (int64_t s = 1; s <= nt && (s == 1 || row_tiles * s <= num_sms()) && (max_split <= 0 || s <= max_split); ++s) {
             const double waves = static_cast<double>(ceil_div(row_tiles * s, num_sms()));
             const double cost = waves * (static_cast<double>(K1) + 128.0 * ceil_div(nt, s));
             if (cost < best_cost * 0.97) { best_cost = cost; best = s; }
@@ -401,11 +401,11 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
 // out may be null (phase 1 only: T is written and nothing else).  All pointers must satisfy tma_ok.
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
-          cudaStream_t stream, const ChainConv* conv) {
+          cudaStream_t stream, const ChainConv* conv, int max_split) {
     ChainPlan plan;
     const int box_h = conv ? conv_box_h(conv->H, conv->W, 128) : 1;
     const int rows_tile = conv ? box_h * conv->W : 128;
-    if (!chain_plan(M, K1, N2, r, out != nullptr, &plan, rows_tile)) return PF_ERR_UNSUPPORTED;
+    if (!chain_plan(M, K1, N2, r, out != nullptr, &plan, rows_tile, max_split)) return PF_ERR_UNSUPPORTED;
     CUtensorMap ta, tb1, tb2, to, tt;
     bool ok = conv ? cached_map_nhwc(&ta, A, conv->N, conv->H, conv->W, conv->C, conv->W, box_h)
                    : cached_map_2d(&ta, A, M, K1, lda, 128);
