@@ -24,9 +24,17 @@
  *     Two calls that may overlap on the GPU must not share a workspace.
  *   - Besides the workspace the library keeps a few fixed device arrays of its own (a
  *     status word and 40 KB of counters at which the thread blocks of a split reduction
- *     meet); calls on different streams of one device may be in flight together: each
- *     launch takes the next of 32 counter sets, so do not keep more than 32 backward
- *     calls of one device unfinished at a time.
+ *     meet).  A reduction over the batch (dU, dV, and x U / dY V when the batch is small) is
+ *     cut into slices whose thread blocks wait for one another inside one launch, so all
+ *     of them must be resident at once: the library sizes such a launch to at most one block
+ *     per SM of the device, which guarantees that on an otherwise idle GPU.  Kernels of
+ *     other streams (or processes) that occupy SMs at the same time can delay a sibling
+ *     block; the wait is bounded (about two seconds), after which the launch gives up, leaves
+ *     its outputs unwritten and pf_last_device_status() reports PF_ERR_TIMEOUT.  Calls of this
+ *     library on different streams of equal priority may be in flight together (each launch
+ *     takes the next of 32 counter sets: keep at most 32 such calls unfinished per device);
+ *     do not mix stream priorities, and do not run backward calls beside long-running
+ *     kernels that pin most SMs.
  *   - Gradients that are sums over the batch (dU, dV) are added in a fixed order:
  *     repeating a call on the same inputs gives bit-identical results.
  *   - Every entry returns a pf_status.  Errors detected on the host (bad pointer,
@@ -102,10 +110,20 @@ int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu
  * Identical to pf_lowrank_linear_fwd except that the scratch is a fixed array inside the
  * library image (PF_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the
  * process exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
- *   - Problems whose pf_lowrank_linear_workspace(m, k, n, r, dtype, 0) exceeds
- *     PF_STATIC_SCRATCH_BYTES are rejected with PF_ERR_WORKSPACE before anything is launched.
- *   - The first call on each device looks up the array's device address (a one-time
- *     set-up with that device current); make that first call outside any stream capture.
+ *   - The bound is the scratch this call will really use, which depends on the path its
+ *     sizes, pointers and pitches select (it can be far below the public workspace query, which
+ *     reserves for every path): many rows at a small rank (m >= 2048, r <= 192, 16-byte aligned
+ *     rows) take the fused kernel, which keeps x U on chip and needs nothing when the stash
+ *     is written directly; otherwise one m x r copy of x U, the fp32 slices of a split first
+ *     product, and re-pitched copies of operands whose row pitch is not a multiple of 16 bytes.
+ *     A call that needs more than PF_STATIC_SCRATCH_BYTES is rejected with PF_ERR_WORKSPACE
+ *     before anything is launched.  Of the benchmark shapes both Transformer-FFN layers fit,
+ *     the LSTM gate layer (700 x 1500 -> 6000, r = 375) fits with 16-byte row pitches and is
+ *     refused with its tight 3000 / 750-byte pitches.
+ *   - The first call on each device is the set-up call: it looks up the array's device address
+ *     with that device current, and (the driver loads modules lazily) it is also when the array
+ *     itself is materialised, so free device memory drops once, by the array's size; no later
+ *     call changes it.  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, which keeps whatever the previous call
  *     left in it: two calls that may overlap on the GPU (different streams) race and must be
  *     ordered by the caller.  Nothing in the array has to be cleared between calls.

@@ -153,27 +153,40 @@ size_t pf_lowrank_linear_workspace(int64_t m, int64_t k, int64_t n, int64_t r, i
     return linear_ws(m, k, n, r, dtype, is_bwd != 0).total;
 }
 
-int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
-                          int64_t ldv, void* y, int64_t ldy, void* T_stash, int64_t ldt,
-                          int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
-                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+}  // extern "C"
+
+namespace pf {
+// The forward behind both entry points.  `exact_need`: instead of the public query's bound (which
+// reserves for every path the call could take), require only the bytes that the path chosen for
+// these pointers will touch; the workspace layout is the same either way.
+int linear_fwd_impl(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
+                    int64_t ldv, void* y, int64_t ldy, void* T_stash, int64_t ldt,
+                    int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream, bool exact_need) {
     int st = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
     if (st != PF_OK) return st;
     if ((!y && m > 0) || ldy < n || !elem_aligned(y, dtype)) return PF_ERR_INVALID_ARG;
     if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
     const LinearWs w = linear_ws(m, k, n, r, dtype, false);
-    st = check_ws(workspace, workspace_bytes, w.total);
-    if (st != PF_OK) return st;
-    if (m == 0) return PF_OK;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
+    tc::LinearArgs a;
+    a.x = x; a.ldx = ldx; a.U = U; a.ldu = ldu; a.V = V; a.ldv = ldv;
+    a.y = y; a.ldy = ldy; a.T = T_stash; a.ldt = ldt;
+    a.m = m; a.k = k; a.n = n; a.r = r;
+    a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.stream = stream;
+    size_t need = w.total;
+    if (exact_need) {
+        bool tc_handles = false;
+        const size_t tc_need = dtype == PF_BF16 ? tc::linear_fwd_need(a, &tc_handles) : 0;
+        if (tc_handles) need = tc_need ? w.off_tc + tc_need : 0;
+        else need = T_stash ? 0 : w.off_T + static_cast<size_t>(m) * r * dtype_size(dtype);   // FMA kernels: x U only
+    }
+    st = check_ws(workspace, workspace_bytes, need);
+    if (st != PF_OK) return st;
+    if (m == 0) return PF_OK;
 
     if (dtype == PF_BF16) {
-        tc::LinearArgs a;
-        a.x = x; a.ldx = ldx; a.U = U; a.ldu = ldu; a.V = V; a.ldv = ldv;
-        a.y = y; a.ldy = ldy; a.T = T_stash; a.ldt = ldt;
-        a.m = m; a.k = k; a.n = n; a.r = r;
-        a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.stream = stream;
         int handled = 0;
         st = tc::linear_fwd(a, &handled);
         if (st != PF_OK || handled) return st;
@@ -183,6 +196,17 @@ int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu
     PF_CUDA(simt_gemm(mk(plainA(x, ldx, 1), plainB(U, ldu, 1), T, ldT, m, r, k, dtype), stream));
     PF_CUDA(simt_gemm(mk(plainA(T, ldT, 1), plainB(V, 1, ldv), y, ldy, m, n, r, dtype), stream));
     return PF_OK;
+}
+}  // namespace pf
+
+extern "C" {
+
+int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
+                          int64_t ldv, void* y, int64_t ldy, void* T_stash, int64_t ldt,
+                          int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return linear_fwd_impl(x, ldx, U, ldu, V, ldv, y, ldy, T_stash, ldt, m, k, n, r, dtype, workspace, workspace_bytes,
+                           cuda_stream, false);
 }
 
 int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,

@@ -99,6 +99,13 @@ cudaError_t repack_rows_bf16_multi(const RepackJob* jobs, int count, cudaStream_
 cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const int64_t* offsets,
                         int count, int elem_bytes, void* flat, cudaStream_t stream);
 
+// The factorized linear forward behind pf_lowrank_linear_fwd and pf_lowrank_linear_fwd_static.
+// exact_need = false: the workspace must satisfy the public query; true: only the bytes the path
+// chosen for these pointers and pitches will touch.
+int linear_fwd_impl(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V, int64_t ldv, void* y,
+                    int64_t ldy, void* T_stash, int64_t ldt, int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream, bool exact_need);
+
 // host-side count of kernels launched by this library
 void count_launch(int n = 1);
 

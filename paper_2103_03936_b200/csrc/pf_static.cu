@@ -39,16 +39,18 @@ extern "C" int pf_lowrank_linear_fwd_static(const void* x, int64_t ldx, const vo
                                             void* cuda_stream) {
     if ((dtype != PF_F32 && dtype != PF_BF16) || m < 0 || k < 1 || n < 1 || r < 1)
         return PF_ERR_INVALID_ARG;
-    const size_t need = pf_lowrank_linear_workspace(m, k, n, r, dtype, 0);
-    if (need > kStaticScratchBytes) return PF_ERR_WORKSPACE;   // problem too large for the fixed scratch
     void* scratch = nullptr;
     const int st = static_scratch(&scratch);
     if (st != PF_OK) return st;
+    // The bound is what this call will really use, not the public workspace query (which reserves for
+    // every path a call of these sizes could take): the fused kernel keeps x U on chip and needs at
+    // most one m x r copy of it, the unfused paths add re-pitched operand copies and fp32 slices.  A
+    // problem that needs more than the array is refused here, before anything is launched.
     // Nothing in the forward reads scratch before writing it (the intermediate x U and the
     // re-pitched operand copies are fully rewritten, pad columns included), so the previous
     // call's contents need no clearing.
-    return pf_lowrank_linear_fwd(x, ldx, U, ldu, V, ldv, y, ldy, T_stash, ldt, m, k, n, r, dtype,
-                                 scratch, kStaticScratchBytes, cuda_stream);
+    return pf::linear_fwd_impl(x, ldx, U, ldu, V, ldv, y, ldy, T_stash, ldt, m, k, n, r, dtype, scratch,
+                               kStaticScratchBytes, cuda_stream, true);
 }
 
 extern "C" size_t pf_static_scratch_bytes(void) { return kStaticScratchBytes; }

@@ -253,8 +253,15 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
         if (ok) {
             const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
             if (p.splits > 1) {
-                float4* blk = reinterpret_cast<float4*>(p.partial) +
-                              (static_cast<size_t>(tile) * p.splits + bz) * (kBM * BN / 4) + (q * 32 + lane);
+                // fp32 slice: this warp's 32 rows go to shared memory as rows of BN floats (the 16-byte
+                // pieces of a row XOR-permuted by the row, which keeps the writes and the later reads
+                // free of bank conflicts), leave as ONE bulk copy of 32 x BN x 4 bytes to the
+                // workspace (the workspace keeps the permuted order; only the sum below reads it),
+                // and the warp reports its arrival once the copy has completed
+                constexpr uint32_t kRowBytes = BN * 4, kPieces = BN / 4;
+                const uint32_t wbase = smem_u32(tiles) + static_cast<uint32_t>(q * 32) * kRowBytes;
+                const uint32_t rbase = wbase + static_cast<uint32_t>(lane) * kRowBytes;
+                const uint32_t rsw = static_cast<uint32_t>(q * 32 + lane) & (kPieces - 1);
 #pragma unroll 1
                 for (int c = 0; c < BN / 32; ++c) {
                     uint32_t v[32];
@@ -262,12 +269,22 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                     tmem_ld_wait();
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
-                        __stcg(blk + (c * 8 + g) * kBM,
-                               make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]),
-                                           __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3])));
+                        st_shared_v4(rbase + (((static_cast<uint32_t>(c * 8 + g)) ^ rsw) << 4),
+                                     make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]));
                 }
-                fence_proxy_async_all();   // the slices are read back by bulk copies (async proxy)
-                __threadfence();
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    uint8_t* dst = reinterpret_cast<uint8_t*>(p.partial) +
+                                   (static_cast<size_t>(tile) * p.splits + bz) * (static_cast<size_t>(kBM) * kRowBytes) +
+                                   static_cast<size_t>(q * 32) * kRowBytes;
+                    bulk_store(dst, wbase, 32u * kRowBytes);
+                    tma_store_commit();
+                    tma_store_wait_all();          // the rows are in the workspace
+                    fence_proxy_async_all();
+                    __threadfence();
+                    atomicAdd(p.counters + 2 * tile, 1u);
+                }
             } else {
                 // every MMA has completed, so the pipeline stages are free: 32 x 33-word panel per warp
                 uint32_t* stg = reinterpret_cast<uint32_t*>(tiles) + (warp - 2) * (32 * 33);
@@ -364,23 +381,24 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     if (warp == 1) tmem_dealloc(tmem_base, BN);
     if (p.splits <= 1) return;
 
-    // ---- slice sum: wait until every slice of this tile is in the workspace, then sum a share of it.
-    // A share is a run of 4-column groups (all 128 rows), contiguous in every slice, so one bulk copy
-    // per slice brings it into the idle pipeline stages: a single trip to L2 for the whole sum.
+    // ---- slice sum: wait until every slice of this tile is in the workspace (four warps of every slice
+    // report), then sum a share of it.  A share is a run of whole rows, contiguous in every slice, so
+    // one bulk copy per slice brings it into the idle pipeline stages: a single trip to L2 for the
+    // whole sum.  The slices are added in slice order (bit-reproducible) and each summed row leaves as
+    // whole 8-byte pieces, a warp writing 256 contiguous bytes per instruction.
     unsigned int* cnt = p.counters + 2 * tile;
     const int S = p.splits;
-    constexpr int kGroups = BN / 4;
-    const int gper = (kGroups + S - 1) / S;
-    const int g_beg = bz * gper;
-    const int ng = max(0, min(kGroups, g_beg + gper) - g_beg);
-    const uint32_t share = static_cast<uint32_t>(ng) * (kBM * 16u);
+    constexpr uint32_t kRowBytes = BN * 4, kPieces = BN / 4;
+    const int rper = (kBM + S - 1) / S;
+    const int r_beg = bz * rper;
+    const int nr = max(0, min(kBM, r_beg + rper) - r_beg);
+    const uint32_t share = static_cast<uint32_t>(nr) * kRowBytes;
     if (threadIdx.x == 0) {
         uint32_t good = (*abort_flag == 0u) ? 1u : 0u;
         if (good) {
-            __threadfence();
-            const unsigned int before = atomicAdd(cnt, 1u);
+            const unsigned int want = 4u * static_cast<unsigned int>(S);
             const long long t0 = clock64();
-            while (before + 1u < static_cast<unsigned int>(S) && ld_acquire_gpu(cnt) < static_cast<unsigned int>(S)) {
+            while (ld_acquire_gpu(cnt) < want) {
                 if (clock64() - t0 > kWaitCycleLimit) {
                     good = 0u;
                     if (p.status) atomicExch(p.status, kStatusTimeout);
@@ -389,14 +407,15 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
             }
             __threadfence();
             fence_proxy_async_all();
-            if (good && ng > 0) {
+            if (good && nr > 0) {
                 const uint32_t bar = smem_u32(&ctl->fix_full);
                 const uint8_t* src = reinterpret_cast<const uint8_t*>(p.partial) +
-                                     (static_cast<size_t>(tile) * S) * (kBM * BN * 4) + static_cast<size_t>(g_beg) * (kBM * 16);
+                                     (static_cast<size_t>(tile) * S) * (static_cast<size_t>(kBM) * kRowBytes) +
+                                     static_cast<size_t>(r_beg) * kRowBytes;
                 mbar_expect_tx(bar, share * static_cast<uint32_t>(S));
                 for (int s = 0; s < S; ++s)
-                    bulk_load(smem_u32(tiles) + static_cast<uint32_t>(s) * share, src + static_cast<size_t>(s) * (kBM * BN * 4),
-                              share, bar);
+                    bulk_load(smem_u32(tiles) + static_cast<uint32_t>(s) * share,
+                              src + static_cast<size_t>(s) * (static_cast<size_t>(kBM) * kRowBytes), share, bar);
                 good = mbar_wait(bar, 0, abort_flag, p.status) ? 1u : 0u;
             }
         }
@@ -405,50 +424,40 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     __syncthreads();
     if (ctl->fix_ok) {
         __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
-        const float4* sm4 = reinterpret_cast<const float4*>(tiles);
-        const uint32_t share4 = share / 16u;
-        // consecutive threads take consecutive rows of one column group: conflict-free 16-byte reads of
-        // shared memory (the other order costs a 5-way bank conflict on every read); each result
-        // leaves as one 8-byte store
+        __nv_bfloat16* C2b = reinterpret_cast<__nv_bfloat16*>(p.C2);
+        const uint32_t base = smem_u32(tiles);
         const bool vec8 = (p.ldc % 4) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 7) == 0;
-        for (int id = threadIdx.x; id < ng * kBM; id += kGemmThreads) {
-            const int gl = id / kBM, rr = id % kBM;
-            float4 acc = sm4[id];
-#pragma unroll 8
+        // consecutive threads take consecutive 16-byte pieces of one row
+        for (int id = threadIdx.x; id < nr * static_cast<int>(kPieces); id += kGemmThreads) {
+            const int rl = id / static_cast<int>(kPieces), pc = id % static_cast<int>(kPieces);
+            const int rr = r_beg + rl;
+            const uint32_t off = static_cast<uint32_t>(rl) * kRowBytes +
+                                 ((static_cast<uint32_t>(pc) ^ (static_cast<uint32_t>(rr) & (kPieces - 1))) << 4);
+            uint4 w = ld_shared_v4(base + off);
+            float4 acc = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
+#pragma unroll 4
             for (int s = 1; s < S; ++s) {
-                const float4 t = sm4[static_cast<uint32_t>(s) * share4 + static_cast<uint32_t>(id)];
-                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+                w = ld_shared_v4(base + static_cast<uint32_t>(s) * share + off);
+                acc.x += __uint_as_float(w.x); acc.y += __uint_as_float(w.y);
+                acc.z += __uint_as_float(w.z); acc.w += __uint_as_float(w.w);
             }
-            const int row = m0 + rr, col = n0 + (g_beg + gl) * 4;
+            const int row = m0 + rr, col = n0 + pc * 4;
             if (row < p.M) {
                 __nv_bfloat16* dst = Cb + static_cast<size_t>(row) * p.ldc + col;
                 if (vec8 && col + 3 < p.N) {
                     *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
-                    continue;
-                }
-                if (col < p.N) dst[0] = __float2bfloat16_rn(acc.x);
-                if (col + 1 < p.N) dst[1] = __float2bfloat16_rn(acc.y);
-                if (col + 2 < p.N) dst[2] = __float2bfloat16_rn(acc.z);
-                if (col + 3 < p.N) dst[3] = __float2bfloat16_rn(acc.w);
-            }
-        }
-        if (p.C2) {   // the same sums once more, for a destination whose pitch the first cannot have
-            __nv_bfloat16* C2b = reinterpret_cast<__nv_bfloat16*>(p.C2);
-            for (int id = threadIdx.x; id < ng * kBM; id += kGemmThreads) {
-                const int gl = id / kBM, rr = id % kBM;
-                float4 acc = sm4[id];
-#pragma unroll 8
-                for (int s = 1; s < S; ++s) {
-                    const float4 t = sm4[static_cast<uint32_t>(s) * share4 + static_cast<uint32_t>(id)];
-                    acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
-                }
-                const int row = m0 + rr, col = n0 + (g_beg + gl) * 4;
-                if (row < p.M) {
-                    __nv_bfloat16* dst = C2b + static_cast<size_t>(row) * p.ldc2 + col;
+                } else {
                     if (col < p.N) dst[0] = __float2bfloat16_rn(acc.x);
                     if (col + 1 < p.N) dst[1] = __float2bfloat16_rn(acc.y);
                     if (col + 2 < p.N) dst[2] = __float2bfloat16_rn(acc.z);
                     if (col + 3 < p.N) dst[3] = __float2bfloat16_rn(acc.w);
+                }
+                if (C2b) {   // the same sums once more, for a destination whose pitch the first cannot have
+                    __nv_bfloat16* d2 = C2b + static_cast<size_t>(row) * p.ldc2 + col;
+                    if (col < p.N) d2[0] = __float2bfloat16_rn(acc.x);
+                    if (col + 1 < p.N) d2[1] = __float2bfloat16_rn(acc.y);
+                    if (col + 2 < p.N) d2[2] = __float2bfloat16_rn(acc.z);
+                    if (col + 3 < p.N) d2[3] = __float2bfloat16_rn(acc.w);
                 }
             }
         }
@@ -690,9 +699,9 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
             bn == 256 || partial == nullptr)
             return PF_ERR_UNSUPPORTED;
         // the slices of a CTA's share are gathered in the pipeline stages
-        const int64_t gper = ceil_div(bn / 4, p.splits);
-        if (gper * p.splits * (kBM * 16) > static_cast<int64_t>(p.num_stages) * (kBM * kBK * 2 + bn * kBK * 2))
-            return PF_ERR_UNSUPPORTED;
+        const int64_t rper = ceil_div(kBM, p.splits);
+        const int64_t room = static_cast<int64_t>(p.num_stages) * (kBM * kBK * 2 + bn * kBK * 2);
+        if (rper * p.splits * (bn * 4) > room || static_cast<int64_t>(kBM) * bn * 4 > room) return PF_ERR_UNSUPPORTED;
         p.counters = next_fix_counters();
         if (!p.counters) return PF_ERR_CUDA;
     }
@@ -766,8 +775,9 @@ int gemm_multi(const GemmLaunch* const* g, int count, cudaStream_t stream) {
         prm[i].num_stages = stages;
         if (i < count) {
             smem = std::max(smem, gemm_smem(src->bn, stages));
-            const int64_t gper = ceil_div(src->bn / 4, prm[i].splits);
-            if (prm[i].splits > 1 && gper * prm[i].splits * (kBM * 16) > static_cast<int64_t>(stages) * (kBM * kBK * 2 + src->bn * kBK * 2))
+            const int64_t rper = ceil_div(kBM, prm[i].splits);
+            const int64_t room = static_cast<int64_t>(stages) * (kBM * kBK * 2 + src->bn * kBK * 2);
+            if (prm[i].splits > 1 && (rper * prm[i].splits * (src->bn * 4) > room || static_cast<int64_t>(kBM) * src->bn * 4 > room))
                 return PF_ERR_UNSUPPORTED;
         }
     }
@@ -855,6 +865,30 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
     const int s1 = std::max(pick_splits(m, r, pick_bn(r), k), bwd ? pick_splits(m, r, pick_bn(r), n) : 1);
     b += align_up(partial_bytes(m, r, s1), 256);
     return b;
+}
+
+// Bytes of `a.ws` that linear_fwd(a) will really touch for these pointers and sizes (it takes the
+// same decisions in the same order), and whether it will handle the call at all.  The public
+// workspace query cannot see pointers and pitches and therefore reserves for every path.
+size_t linear_fwd_need(const LinearArgs& a, bool* handles) {
+    *handles = false;
+    if (encode_fn() == nullptr) return 0;
+    if (a.k > (1 << 22) || a.n > (1 << 22) || a.r > (1 << 22)) return 0;
+    size_t room = 0;
+    const struct { const void* p; int64_t ld, rows, cols; } ops[3] = {
+        {a.x, a.ldx, a.m, a.k}, {a.U, a.ldu, a.k, a.r}, {a.V, a.ldv, a.n, a.r}};
+    for (const auto& o : ops) {
+        if (tma_ok(o.p, o.ld)) continue;
+        if (o.cols % 8 == 0) return 0;               // declined: FMA kernels
+        room += repack_room(o.rows, o.cols);
+    }
+    *handles = true;
+    const size_t t_bytes = align_up(static_cast<size_t>(a.m) * pad8(a.r) * 2, 256);
+    const bool stash_direct = a.T && tma_ok(a.T, a.ldt);
+    ChainPlan plan;
+    if (use_chain(a.m, a.r) && tma_ok(a.y, a.ldy) && chain_plan(a.m, a.k, a.n, a.r, true, &plan))
+        return room + ((a.T && !stash_direct) ? t_bytes : 0);
+    return room + t_bytes + align_up(partial_bytes(a.m, a.r, pick_splits(a.m, a.r, pick_bn(a.r), a.k)), 256);
 }
 
 int linear_fwd(const LinearArgs& a, int* handled) {
@@ -966,8 +1000,32 @@ int linear_bwd(const LinearArgs& a, int* handled) {
                    dv_beside ? 1 : 0);
         if (st != PF_OK) return st;
     } else {
-        st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG,
-                  pick_splits(a.m, a.r, pick_bn(a.r), a.n), p1, a.stream);
+        // Few rows: G = dY V is a contraction split across blocks, and dV = dY^T T, which needs nothing
+        // of it, shares its launch (the second block slot of every SM); dU and dX follow in a second one.
+        const int sg = pick_splits(a.m, a.r, pick_bn(a.r), a.n);
+        GemmLaunch gg, gv, gu, gx;
+        bool ok = !pair_worthwhile(a.m, a.r, a.n) && !pair_worthwhile(a.n, a.r, a.m) &&
+                  gemm_prepare({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG, sg, p1, nullptr, &gg) == PF_OK &&
+                  gemm_prepare({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, nullptr, &gv) == PF_OK &&
+                  gemm_prepare({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, nullptr, &gu) == PF_OK;
+        if (ok && a.dX)
+            ok = gemm_prepare({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, nullptr, &gx) == PF_OK;
+        ok = ok && (gg.p.splits > 1 || gv.p.splits <= 1) && (gu.p.splits > 1 || !a.dX || gx.p.splits <= 1);
+        if (ok) {
+            const GemmLaunch* first[2] = {&gg, &gv};
+            st = gemm_multi(first, 2, a.stream);
+            if (st == PF_OK) {
+                const GemmLaunch* second[2] = {&gu, &gx};
+                st = gemm_multi(second, a.dX ? 2 : 1, a.stream);
+                if (st != PF_ERR_UNSUPPORTED) return st;
+                // tile widths that cannot share a launch: one launch each
+                st = launch_prepared(gu, a.stream);
+                if (st == PF_OK && a.dX) st = launch_prepared(gx, a.stream);
+                return st;
+            }
+            if (st != PF_ERR_UNSUPPORTED) return st;
+        }
+        st = gemm({dY.p, dY.ld, false}, {V.p, V.ld, true}, a.m, a.r, a.n, G, ldG, sg, p1, a.stream);
         if (st != PF_OK) return st;
         dx_pending = a.dX != nullptr;
     }

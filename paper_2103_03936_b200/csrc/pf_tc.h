@@ -56,6 +56,7 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
 size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
                             int pad, bool bwd);
 void reset_fix_counters();  // clears the slice-sum counters (after PF_ERR_TIMEOUT)
+size_t linear_fwd_need(const LinearArgs& a, bool* handles);   // bytes of a.ws the forward really touches
 int linear_fwd(const LinearArgs& a, int* handled);
 int linear_bwd(const LinearArgs& a, int* handled);
 int conv_fwd(const ConvArgs& a, int* handled);

@@ -74,14 +74,53 @@ def test_static_scratch_forward_without_stash_uses_the_array_for_the_intermediat
         _check(case, stash=False)
 
 
+def test_which_benchmark_shapes_fit_the_array():
+    """The bound is what the chosen path really uses.  The Transformer-FFN shapes take the fused
+    kernel (x U stays on chip, the stash is written directly): they fit.  The LSTM shape fits with
+    16-byte row pitches (x U once plus the fp32 slices of the split first product, 7.4 MiB) and is
+    refused with the tight pitches of 3000 / 750 bytes, whose re-pitched copies of x, U and V alone
+    take 7.7 MiB."""
+    _first_call_on_this_device()
+    for name in ("C2a", "C2b"):
+        c = wl.linear_cases()[name]
+        d = c.generate()
+        x, U, V = (dev(d[k_], c.dtype) for k_ in ("x", "U", "V"))
+        y_ref, T_ref = pf.pf_lowrank_linear_fwd(x, U, V, want_stash=True)
+        y, T = torch.empty_like(y_ref), torch.empty_like(T_ref)
+        pf.pf_lowrank_linear_fwd_static(x, U, V, y=y, T_stash=T)
+        torch.cuda.synchronize()
+        assert torch.equal(y, y_ref) and torch.equal(T, T_ref), name
+    c = wl.linear_cases()["C3i"]
+    d = c.generate()
+
+    def padded(a, cols, ld):
+        buf = torch.zeros((a.shape[0], ld), dtype=torch.bfloat16, device="cuda")
+        buf[:, :cols] = dev(a, c.dtype)
+        return buf[:, :cols]
+    x, U, V = padded(d["x"], 1500, 1504), padded(d["U"], 375, 376), padded(d["V"], 375, 376)
+    y_ref = pf.pf_lowrank_linear_fwd(x, U, V)
+    y = torch.empty_like(y_ref)
+    pf.pf_lowrank_linear_fwd_static(x, U, V, y=y)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y_ref)
+    xt, Ut, Vt = (dev(d[k_], c.dtype) for k_ in ("x", "U", "V"))       # tight pitches
+    before = pf.pf_launch_count()
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_lowrank_linear_fwd_static(xt, Ut, Vt, y=y)
+    assert e.value.status == 3 and pf.pf_launch_count() == before
+    assert pf.pf_last_device_status() == 0
+
+
 def test_problem_larger_than_the_array_is_refused_before_any_launch():
     assert pf.pf_static_scratch_bytes() == 8 << 20
-    m, k, n, r = 1 << 20, 64, 64, 64          # needs far more than the array for x U alone
-    assert pf.pf_lowrank_linear_workspace(m, k, n, r, pf.PF_BF16, 0) > pf.pf_static_scratch_bytes()
-    x = torch.empty((8, k), dtype=torch.bfloat16, device="cuda")       # never dereferenced
-    U = torch.empty((k, r), dtype=torch.bfloat16, device="cuda")
-    V = torch.empty((n, r), dtype=torch.bfloat16, device="cuda")
+    m, k, n, r = 2000, 64, 64, 4096           # few rows: unfused products, and x U alone is 16 MB
+    assert m * r * 2 > pf.pf_static_scratch_bytes()
+    # real buffers of the right sizes: were the call accepted by mistake, it would still stay in bounds
+    x = torch.zeros((m, k), dtype=torch.bfloat16, device="cuda")
+    U = torch.zeros((k, r), dtype=torch.bfloat16, device="cuda")
+    V = torch.zeros((n, r), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((m, n), dtype=torch.bfloat16, device="cuda")
     before = pf.pf_launch_count()
-    st = pf.lib().pf_lowrank_linear_fwd_static(x.data_ptr(), k, U.data_ptr(), r, V.data_ptr(), r,
-                                               x.data_ptr(), n, None, 0, m, k, n, r, pf.PF_BF16, None)
-    assert st == 3 and pf.pf_launch_count() == before
+    with pytest.raises(pf.PfError) as e:
+        pf.pf_lowrank_linear_fwd_static(x, U, V, y=y)
+    assert e.value.status == 3 and pf.pf_launch_count() == before
