@@ -97,7 +97,7 @@ def _floors(flops_fwd, bytes_fwd, bytes_bwd, pk):
     return f, b
 
 
-def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32):
+def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32, library=True, repeats=5):
     tdt = torch.bfloat16 if dtype == wl.BF16 else torch.float32
     s = 2 if dtype == wl.BF16 else 4
     code = pf.PF_BF16 if dtype == wl.BF16 else pf.PF_F32
@@ -127,13 +127,13 @@ def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32):
     for c in sets[0]:
         c()
     launches = pf.pf_launch_count() - l0
-    t = _time(sets, iters)
+    t = _time(sets, iters, repeats=repeats)
     flops_fwd = 2.0 * m * r * (k + n)
     bytes_fwd = s * (m * k + m * n + r * (k + n))
     bytes_bwd = s * (m * n + 2 * m * k + 2 * r * (k + n))
     ff, fb = _floors(flops_fwd, bytes_fwd, bytes_bwd, pk)
     tot = t[-1]["median_us"]
-    lib = _library_linear(lib_sets, U, V, iters)
+    lib = _library_linear(lib_sets, U, V, iters) if library else (None, None, None)
     return {"config": name, "kind": "linear", "m": m, "k": k, "n": n, "r": r, "dtype": dtype,
             "library_fwd_us": lib[0], "library_bwd_us": lib[1], "library_fwd_bwd_us": lib[2],
             "pitch": "padded to 16 B" if pad_pitch else "tight", "buffer_sets": nsets, "launches_fwd_bwd": launches,
@@ -142,7 +142,7 @@ def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32):
             "tflops": 3 * flops_fwd / tot / 1e6, "gbs": (bytes_fwd + bytes_bwd) / tot / 1e3}
 
 
-def conv_config(name, c, pk, iters=20):
+def conv_config(name, c, pk, iters=20, repeats=5):
     tdt = torch.bfloat16
     M = c.N * c.H * c.W
     foot = 2 * (2 * M * c.C + 2 * M * c.O + M * c.R)
@@ -171,7 +171,7 @@ def conv_config(name, c, pk, iters=20):
     for cc in sets[0]:
         cc()
     launches = pf.pf_launch_count() - l0
-    t = _time(sets, iters)
+    t = _time(sets, iters, repeats=repeats)
     Keff = c.kh * c.kw * c.C
     flops_fwd = 2.0 * M * c.R * (Keff + c.O)
     bytes_fwd = 2 * (M * c.C + M * c.O + c.R * (Keff + c.O))
@@ -201,6 +201,30 @@ def pack_config(name, numels, pk, iters=30):
     us = t[0]["median_us"]
     return {"config": name, "kind": "pack", "tensors": len(numels), "elements": total, "dtype": "bf16",
             "us": us, "gbs": 4.0 * total / us / 1e3, "roofline_frac": (4.0 * total / (pk["hbm_gbs"] * 1e9) * 1e6) / us}
+
+
+def quick(pk):
+    """The configurations the roofline target names, timed with the same back-to-back protocol but few
+    repetitions (a few seconds in all), for the benchmark's JSON line: per configuration the forward,
+    the backward and the pair in microseconds, the roofline floor and the fraction reached."""
+    out = {}
+
+    def keep(r):
+        out[r["config"] + (" (16 B pitches)" if r.get("pitch") == "padded to 16 B" else "")] = {
+            "fwd_us": round(r["fwd_us"], 2), "bwd_us": round(r["bwd_us"], 2), "fwd_bwd_us": round(r["fwd_bwd_us"], 2),
+            "floor_us": round(r["floor_fwd_us"] + r["floor_bwd_us"], 2), "roofline_frac": round(r["roofline_frac"], 4),
+            "launches": r.get("launches_fwd_bwd", r.get("launches_fwd_bwd_pack"))}
+
+    keep(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk, iters=24, library=False, repeats=3))
+    keep(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk, iters=24, library=False, repeats=3))
+    keep(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, iters=24, library=False, repeats=3))
+    keep(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True, iters=24, library=False, repeats=3))
+    for name, c in wl.conv_cases().items():
+        keep(conv_config(f"{name} conv", c, pk, iters=8, repeats=3))
+    for r in (128, 512):
+        keep(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=6, library=False, repeats=3))
+        torch.cuda.empty_cache()
+    return out
 
 
 def run(path, pk, only=None):
