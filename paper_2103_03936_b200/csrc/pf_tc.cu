@@ -137,6 +137,22 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     // it does not wait for that kernel: its blocks run beside it on SMs that kernel leaves free.  (Every
     // kernel of this library lets its successor start only after its own wait has returned, i.e. once
     // everything older in the stream is complete, so older results are safe to read.)
+    // While the previous kernel of the stream finishes, ask L2 for this block's first tiles (a prefetch
+    // only moves lines into L2, the point of coherence: harmless even if that kernel still writes them).
+    if (p.conv_mode == 0 && (warp == 0 || warp == 6) && elect_one()) {
+        for (int i = 0; i < 6 && i < nkb; ++i) {
+            const int k0 = (kb_beg + i) * kBK;
+            if (warp == 0) {
+                if (p.a_mn) { tma_prefetch_l2_2d(&tmA, m0, k0); tma_prefetch_l2_2d(&tmA, m0 + 64, k0); }
+                else tma_prefetch_l2_2d(&tmA, k0, m0);
+            } else if (p.b_mn) {
+#pragma unroll
+                for (int h = 0; h < BN / 64; ++h) tma_prefetch_l2_2d(&tmB, n0 + 64 * h, k0);
+            } else {
+                tma_prefetch_l2_2d(&tmB, k0, n0);
+            }
+        }
+    }
     if (!p.independent) pdl_wait();     // everything above overlapped the previous kernel's tail
     pdl_launch_dependents();
     const uint32_t tmem_base = ctl->tmem_base;
@@ -608,27 +624,35 @@ void pick_pair_splits(int64_t Mu, int64_t Mv, int64_t N, int64_t K, int kblock, 
 }
 
 // Slices of dU (k x r) and dV (n x r) in the backward of the linear layer, and whether dV runs BESIDE
-// the fused dX kernel instead of after it.  dV = dY^T T needs nothing that kernel writes.  When the
-// contraction of its first product is long against its output (n >= 2k), the fused kernel is left
-// unsplit (one block per 128-row tile, no block repeats another's first product), which leaves SMs
-// free; the dV blocks are sized to exactly those SMs and do not wait for the fused kernel, and the
-// dU blocks (which need G) follow on the SMs the fused kernel vacates.
-void bwd_split_plan(int64_t m, int64_t k, int64_t n, int64_t r, bool fused_dx, int* su, int* sv, bool* beside) {
+// the fused dX kernel instead of after it.  dV = dY^T T needs nothing that kernel writes, so when the
+// fused kernel leaves at least one SM per dV tile free, the dV blocks are sized to exactly those SMs,
+// come first in their launch and do not wait for the fused kernel; the dU blocks (which need G)
+// follow on the other SMs once that kernel's blocks retire.  When the contraction of the fused kernel's
+// first product is long against its output (n >= 2k) it is left unsplit for this (`unsplit`: one
+// block per 128-row tile, no block repeats another's first product), which frees more SMs.
+// `fused_blocks` = blocks of the fused kernel with the column split it would choose by itself, 0 = no
+// fused kernel.
+void bwd_split_plan(int64_t m, int64_t k, int64_t n, int64_t r, int64_t fused_blocks, int* su, int* sv, bool* beside,
+                    bool* unsplit) {
     pick_pair_splits(k, n, r, m, kBK, su, sv);
     *beside = false;
-    if (!fused_dx || n < 2 * k) return;
+    *unsplit = false;
+    if (fused_blocks <= 0) return;
     const int bn = pick_bn(r);
     const int64_t row_tiles = ceil_div(m, kBM), nkb = ceil_div(m, kBK);
     const int64_t tu = ceil_div(k, kBM) * ceil_div(r, bn), tv = ceil_div(n, kBM) * ceil_div(r, bn);
-    const int64_t free_sms = num_sms() - row_tiles;
+    const bool force = n >= 2 * k;
+    const int64_t free_sms = num_sms() - (force ? row_tiles : fused_blocks);
     const int64_t smax = std::max<int64_t>(1, std::min<int64_t>(64, nkb / 4));
-    if (free_sms < tv || tu + tv > num_sms()) return;
+    if (free_sms < tv || tu > num_sms() || tu > kFixTiles || tv > kFixTiles) return;
     const int64_t b = std::min(free_sms / tv, smax);
+    // dU gets the SMs that dV does not hold: dV may still be running when the fused kernel retires
     const int64_t a = std::min((num_sms() - tv * b) / tu, smax);
     if (a < 1 || b < 1) return;
     *su = static_cast<int>(a);
     *sv = static_cast<int>(b);
     *beside = true;
+    *unsplit = force;
 }
 
 // C[M,N] (bf16, ldc) = A * B.  `partial` must hold splits*M*N floats when splits > 1.
@@ -765,13 +789,19 @@ int gemm_multi(const GemmLaunch* const* g, int count, cudaStream_t stream) {
             seen_plain = true;
         }
     }
-    if (split_ctas > num_sms()) return PF_ERR_UNSUPPORTED;
+    // The blocks of a split product wait for one another and must be resident together.  A first
+    // product marked independent never waits for anything later in the launch and is dispatched
+    // first, so it only has to fit by itself, and the products behind it by themselves.
+    const bool lead = count > 1 && g[0]->p.independent && g[0]->p.splits > 1;
+    const int resident = lead ? std::max(ctas[0], split_ctas - ctas[0]) : split_ctas;
+    if (resident > num_sms()) return PF_ERR_UNSUPPORTED;
+    const int wave = lead ? std::max(ctas[0], total - ctas[0]) : total;
     GemmParams prm[3];
     size_t smem = 0;
     for (int i = 0; i < 3; ++i) {
         const GemmLaunch* src = g[i < count ? i : 0];
         prm[i] = src->p;
-        const int stages = pick_stages(src->bn, total);
+        const int stages = pick_stages(src->bn, wave);
         prm[i].num_stages = stages;
         if (i < count) {
             smem = std::max(smem, gemm_smem(src->bn, stages));
@@ -841,6 +871,25 @@ size_t repack_room(int64_t rows, int64_t cols) {
     return cols % 8 == 0 ? 0 : align_up(static_cast<size_t>(rows) * pad8(cols) * 2, 256);
 }
 
+// Room for the fp32 slices of dU and dV under either backward structure (which one a call takes
+// depends on pointers the workspace query does not see): no block count exceeds one per SM per product.
+void bwd_partial_bytes(int64_t m, int64_t k, int64_t n, int64_t r, size_t* bytes_u, size_t* bytes_v) {
+    int su, sv;
+    bool beside, unsplit;
+    bwd_split_plan(m, k, n, r, 0, &su, &sv, &beside, &unsplit);
+    size_t bu = partial_bytes(k, r, su), bv = partial_bytes(n, r, sv);
+    ChainPlan plan;
+    if (use_chain(m, r) && chain_plan(m, n, k, r, true, &plan)) {
+        for (int64_t fused_blocks : {static_cast<int64_t>(plan.row_tiles) * plan.nsplit, static_cast<int64_t>(plan.row_tiles)}) {
+            bwd_split_plan(m, k, n, r, fused_blocks, &su, &sv, &beside, &unsplit);
+            bu = std::max(bu, partial_bytes(k, r, su));
+            bv = std::max(bv, partial_bytes(n, r, sv));
+        }
+    }
+    *bytes_u = align_up(bu, 256);
+    *bytes_v = align_up(bv, 256);
+}
+
 }  // namespace
 
 // Extra workspace of the tensor-core linear path: repack buffers for operands whose width is not a
@@ -854,12 +903,9 @@ size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool b
         b += repack_room(m, n);                                             // dY
         b += align_up(static_cast<size_t>(m) * pad8(r) * 2, 256);           // G at padded pitch
         // slices for either backward structure (the choice depends on pointers the query does not see)
-        int su, sv, su2, sv2;
-        bool beside;
-        bwd_split_plan(m, k, n, r, false, &su, &sv, &beside);
-        bwd_split_plan(m, k, n, r, true, &su2, &sv2, &beside);
-        b += align_up(std::max(partial_bytes(k, r, su), partial_bytes(k, r, su2)), 256) +
-             align_up(std::max(partial_bytes(n, r, sv), partial_bytes(n, r, sv2)), 256);
+        size_t bu, bv;
+        bwd_partial_bytes(m, k, n, r, &bu, &bv);
+        b += bu + bv;
     }
     // skinny batches: the m x r products (x U, dY V) are split over their contraction to fill the SMs
     const int s1 = std::max(pick_splits(m, r, pick_bn(r), k), bwd ? pick_splits(m, r, pick_bn(r), n) : 1);
@@ -971,18 +1017,10 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     const bool fused_dx = use_chain(a.m, a.r) && (!a.dX || tma_ok(a.dX, a.lddx)) &&
                           chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan);
     int su, sv;
-    bool dv_beside;
-    bwd_split_plan(a.m, a.k, a.n, a.r, fused_dx, &su, &sv, &dv_beside);
-    {   // the workspace holds room for the slices of either structure (see linear_extra_workspace)
-        int s0, s1, s2, s3;
-        bool unused;
-        bwd_split_plan(a.m, a.k, a.n, a.r, false, &s0, &s1, &unused);
-        bwd_split_plan(a.m, a.k, a.n, a.r, true, &s2, &s3, &unused);
-        const size_t bu = std::max(partial_bytes(a.k, a.r, s0), partial_bytes(a.k, a.r, s2));
-        const size_t bv = std::max(partial_bytes(a.n, a.r, s1), partial_bytes(a.n, a.r, s3));
-        pu_bytes = align_up(bu, 256);
-        pv_bytes = align_up(bv, 256);
-    }
+    bool dv_beside, chain_unsplit;
+    bwd_split_plan(a.m, a.k, a.n, a.r, fused_dx ? static_cast<int64_t>(plan.row_tiles) * plan.nsplit : 0, &su, &sv, &dv_beside,
+                   &chain_unsplit);
+    bwd_partial_bytes(a.m, a.k, a.n, a.r, &pu_bytes, &pv_bytes);
     float* pu = reinterpret_cast<float*>(scratch);
     scratch += pu_bytes;
     float* pv = reinterpret_cast<float*>(scratch);
@@ -997,7 +1035,7 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     bool dx_pending = false;     // dX still to be computed as a plain product G U^T
     if (fused_dx) {
         st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream, nullptr,
-                   dv_beside ? 1 : 0);
+                   chain_unsplit ? 1 : 0);
         if (st != PF_OK) return st;
     } else {
         // Few rows: G = dY V is a contraction split across blocks, and dV = dY^T T, which needs nothing

@@ -33,6 +33,7 @@ constexpr int kMaxStages = 8;
 constexpr int kChainThreads = 352;          // A producer, MMA warp, 8 epilogue warps, B producer
 constexpr uint32_t kTileBytes = 16384;      // 128 rows x 64 bf16
 constexpr int kAccBufs = 4;                 // 4 x 128 TMEM columns of phase-2 accumulators
+constexpr int kEarlyTiles = 8;              // tiles of A requested into L2 before the dependency wait
 
 struct ChainCtl {
     uint64_t full[kMaxStages];
@@ -124,6 +125,17 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // While the previous kernel of the stream finishes, ask L2 for this block's first tiles.  A prefetch
+    // only moves lines into L2, the point of coherence, so it is harmless even if that kernel is
+    // still writing the tensor; the loads that consume the data are issued after the wait below.
+    if (p.conv_cblks == 0) {
+        if (warp == 0 && elect_one()) {
+            for (int kb = 0; kb < kEarlyTiles && kb < nkb1; ++kb) tma_prefetch_l2_2d(&tmA, kb * 64, m0);
+        } else if (warp == 10 && elect_one()) {
+            for (int kb = 0; kb < 2 && kb < nkb1; ++kb)
+                for (int q = 0; q < nkb2; ++q) tma_prefetch_l2_2d(&tmB1, q * 64, kb * 64);
+        }
+    }
     pdl_wait();                 // everything above overlapped the previous kernel's tail
     pdl_launch_dependents();
     const uint32_t tmem = ctl->tmem_base;
