@@ -185,7 +185,7 @@ def conv_config(name, c, pk, iters=20, repeats=5):
             "tflops": 3 * flops_fwd / tot / 1e6, "gbs": (bytes_fwd + bytes_bwd) / tot / 1e3}
 
 
-def pack_config(name, numels, pk, iters=30):
+def pack_config(name, numels, pk, iters=30, repeats=5):
     tdt = torch.bfloat16
     grads = [torch.randn(n, device="cuda").to(tdt) for n in numels]
     total = sum(numels)
@@ -197,7 +197,7 @@ def pack_config(name, numels, pk, iters=30):
         flat = torch.empty(total, dtype=tdt, device="cuda")
         call, _ = pf.pf_pack_factor_grads(g, flat=flat, stream=stream, prepare=True)
         sets.append((call,))
-    t = _time(sets, iters)
+    t = _time(sets, iters, repeats=repeats)
     us = t[0]["median_us"]
     return {"config": name, "kind": "pack", "tensors": len(numels), "elements": total, "dtype": "bf16",
             "us": us, "gbs": 4.0 * total / us / 1e3, "roofline_frac": (4.0 * total / (pk["hbm_gbs"] * 1e9) * 1e6) / us}
@@ -227,8 +227,10 @@ def quick(pk):
     return out
 
 
-def run(path, pk, only=None):
-    """only: optional substring; configurations whose name lacks it are skipped."""
+def run(path, pk, only=None, iters=None, repeats=5, library=True):
+    """only: optional substring; configurations whose name lacks it are skipped.  iters / repeats /
+    library: fewer back-to-back calls per batch, fewer batches, no library comparison (the short
+    form a profiler wraps)."""
     rows = []
 
     def emit(r):
@@ -239,26 +241,60 @@ def run(path, pk, only=None):
             for rr in rows:
                 f.write(json.dumps(rr) + "\n")
 
+    def it(default):
+        return default if iters is None else iters
+
     want = (lambda nm: only is None or only in nm)
+    lin = dict(library=library, repeats=repeats)
     if want("C1 tiny fp32"):
-        emit(linear_config("C1 tiny fp32", 64, 256, 256, 32, wl.F32, pk))
+        emit(linear_config("C1 tiny fp32", 64, 256, 256, 32, wl.F32, pk, iters=it(32), **lin))
     if want("C2a FFN up"):
-        emit(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk))
+        emit(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk, iters=it(32), **lin))
     if want("C2b FFN down"):
-        emit(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk))
-    if want("C3 LSTM gates"):
-        emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk))
-    if want("C3 LSTM gates"):
-        emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True))
+        emit(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk, iters=it(32), **lin))
+    if want("C3 LSTM gates tight"):
+        emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, iters=it(32), **lin))
+    if want("C3 LSTM gates padded"):
+        emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True, iters=it(32), **lin))
     for name, c in wl.conv_cases().items():
         if want(f"{name} conv"):
-            emit(conv_config(f"{name} conv", c, pk))
+            emit(conv_config(f"{name} conv", c, pk, iters=it(20), repeats=repeats))
     for r in wl.SWEEP_RANKS:
         if want(f"C5 sweep r={r}"):
-            emit(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=8))
+            emit(linear_config(f"C5 sweep r={r}", 16384, 4096, 4096, r, wl.BF16, pk, iters=it(8), **lin))
+            torch.cuda.empty_cache()
     # ResNet-18-sized and Transformer-sized factor-gradient lists (Table 4 / Table 3 parameter counts)
     if want("pack ~3.3M elements"):
-        emit(pack_config("pack ~3.3M elements", [147457, 16384, 589821, 65536, 1179653, 131072, 1179648, 131071], pk))
+        emit(pack_config("pack ~3.3M elements", [147457, 16384, 589821, 65536, 1179653, 131072, 1179648, 131071], pk,
+                         iters=it(30), repeats=repeats))
     if want("pack ~26.7M elements"):
-        emit(pack_config("pack ~26.7M elements", [65536 + (i % 3) for i in range(100)] + [262144 - (i % 5) for i in range(76)], pk))
+        emit(pack_config("pack ~26.7M elements", [65536 + (i % 3) for i in range(100)] + [262144 - (i % 5) for i in range(76)], pk,
+                         iters=it(30), repeats=repeats))
     return rows
+
+
+def main():
+    """`python bench_suite.py --only "C4 conv" --iters 2`: time (and thereby launch) one or a few
+    configurations by themselves, e.g. as the small command a profiler wraps."""
+    import argparse
+    import os
+    import sys
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--only", required=True, help="substring of the configuration names to run")
+    ap.add_argument("--out", default=os.devnull, help="file for the JSON lines")
+    ap.add_argument("--iters", type=int, default=None, help="back-to-back calls per timed batch")
+    ap.add_argument("--repeats", type=int, default=5, help="timed batches per call")
+    ap.add_argument("--no-library", action="store_true", help="skip the library (cuBLAS) comparison")
+    args = ap.parse_args()
+    root = os.path.dirname(os.path.abspath(__file__))
+    if root not in sys.path:
+        sys.path.insert(0, root)
+    import bench
+    torch.cuda.set_device(0)
+    for row in run(args.out, bench.peaks(), only=args.only, iters=args.iters, repeats=args.repeats,
+                   library=not args.no_library):
+        print(json.dumps(row))
+
+
+if __name__ == "__main__":
+    main()
