@@ -151,6 +151,52 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------
+ * Grouped factorized fully-connected layers: `groups` layers of ONE shape (m, k, n, r), each with its
+ * own factor pair (U_g, V_g), in one call -- the per-gate factorization of an LSTM layer
+ * (Section 2.3, eq. "lr-lstm-rule": every gate matrix W_i*, W_h* is replaced by its own U V^T; the
+ * LSTM table of the appendix lists the 1500 x 375 / 375 x 1500 factors per gate) and the four
+ * projections W^Q, W^K, W^V, W^O of a factorized attention block (Section 2.4).
+ *     y_g = (x_g U_g) V_g^T ,   g = 0 .. groups-1
+ * Every tensor of group g starts s* ELEMENTS after that of group g-1 (sx for x, su for U, ...); the
+ * matrices themselves are as in the ungrouped calls.  sx = 0 means ONE input x shared by all groups
+ * (the gates of an LSTM all read the same x_t); factors and outputs are always per group.
+ * With bf16 and 16-byte aligned pointers, pitches and strides the whole call is two launches
+ * (all x_g U_g, then all T_g V_g^T), whatever `groups`; other layouts, and fp32, run group by group
+ * through the ungrouped kernels (same results, more launches).
+ *
+ * Backward, for dY_g [m, n] (stride sdy):
+ *   dU_g = x_g^T (dY_g V_g),  dV_g = dY_g^T (x_g U_g)                       (strides sdu, sdv)
+ *   dX_g = (dY_g V_g) U_g^T   (stride sdx)            when every group has its own x (sx != 0);
+ *   dX   = sum over g of (dY_g V_g) U_g^T, ONE m x k matrix (sdx ignored)   when x is shared (sx = 0),
+ *          since a shared input collects the gradient of every group that reads it.
+ *   NULL dX = not wanted.  T_stash (stride st): the forward's stash, or NULL to recompute.
+ * Two launches (three when T is recomputed) on the fast path.
+ * ------------------------------------------------------------------------------- */
+size_t pf_lowrank_linear_grouped_workspace(int groups, int64_t m, int64_t k, int64_t n, int64_t r,
+                                           int dtype, int is_bwd);
+
+int pf_lowrank_linear_grouped_fwd(int groups,
+                                  const void* x, int64_t ldx, int64_t sx,
+                                  const void* U, int64_t ldu, int64_t su,
+                                  const void* V, int64_t ldv, int64_t sv,
+                                  void* y, int64_t ldy, int64_t sy,
+                                  void* T_stash, int64_t ldt, int64_t st,
+                                  int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+int pf_lowrank_linear_grouped_bwd(int groups,
+                                  const void* x, int64_t ldx, int64_t sx,
+                                  const void* U, int64_t ldu, int64_t su,
+                                  const void* V, int64_t ldv, int64_t sv,
+                                  const void* dY, int64_t lddy, int64_t sdy,
+                                  const void* T_stash, int64_t ldt, int64_t st,
+                                  void* dX, int64_t lddx, int64_t sdx,
+                                  void* dU, int64_t lddu, int64_t sdu,
+                                  void* dV, int64_t lddv, int64_t sdv,
+                                  int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------
  * Factorized convolution: a kh x kw convolution into R channels (factor U) followed by a
  * 1 x 1 convolution to O channels (factor V), nothing in between
  * (Section 2.2 "Factorizing a convolution layer"; Appendix B "Convolution layer").

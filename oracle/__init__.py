@@ -10,6 +10,7 @@ Functions (paper passages they follow are cited in ``pf_oracle.c``):
 
     linear_fwd(x, U, V)              -> y, T            y = (x U) V^T
     linear_bwd(x, U, V, dY)          -> dX, dU, dV      chain rule on the above
+    linear_grouped_fwd / _bwd(x, U, V[, dY])            the same for G factor pairs (shared or own x)
     conv_fwd(x, U, V, stride, pad)   -> y, T            k x k conv to r channels, then 1 x 1
     conv_bwd(x, U, V, dY, stride, pad) -> dX, dU, dV
     pack(list_of_arrays)             -> flat, offsets   flat gradient buffer
@@ -105,6 +106,25 @@ def linear_bwd(x, U, V, dY):
     _load().pf_oracle_linear_bwd(_p(x), _p(U), _p(V), _p(dY), _p(T), m, k, n, r,
                                  _p(G), _p(dX), _p(dU), _p(dV))
     return dX, dU, dV
+
+
+def linear_grouped_fwd(x, U, V):
+    """Grouped layer (Section 2.3, per-gate LSTM factors; Section 2.4, attention projections):
+    y[g] = (x[g] U[g]) V[g]^T for every group g, each through linear_fwd.  x is [G, m, k], or
+    [m, k] when all groups read the same input."""
+    G = len(U)
+    out = [linear_fwd(x if np.ndim(x) == 2 else x[g], U[g], V[g]) for g in range(G)]
+    return np.stack([o[0] for o in out]), np.stack([o[1] for o in out])
+
+
+def linear_grouped_bwd(x, U, V, dY):
+    """Gradients of the grouped layer, group by group through linear_bwd.  An input shared by all
+    groups collects the gradient of every group that reads it: dX = sum over g of dX[g]."""
+    G = len(U)
+    shared = np.ndim(x) == 2
+    out = [linear_bwd(x if shared else x[g], U[g], V[g], dY[g]) for g in range(G)]
+    dX = np.sum([o[0] for o in out], axis=0) if shared else np.stack([o[0] for o in out])
+    return dX, np.stack([o[1] for o in out]), np.stack([o[2] for o in out])
 
 
 def conv_out_hw(H, W, kh, kw, stride, pad):

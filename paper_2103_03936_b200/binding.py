@@ -52,6 +52,12 @@ def lib() -> ctypes.CDLL:
         L.pf_lowrank_linear_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                             vp, i64, vp, i64, vp, i64,
                                             i64, i64, i64, i64, ci, vp, sz, vp]
+        L.pf_lowrank_linear_grouped_workspace.restype = sz
+        L.pf_lowrank_linear_grouped_workspace.argtypes = [ci, i64, i64, i64, i64, ci, ci]
+        L.pf_lowrank_linear_grouped_fwd.restype = ci
+        L.pf_lowrank_linear_grouped_fwd.argtypes = [ci] + [vp, i64, i64] * 5 + [i64, i64, i64, i64, ci, vp, sz, vp]
+        L.pf_lowrank_linear_grouped_bwd.restype = ci
+        L.pf_lowrank_linear_grouped_bwd.argtypes = [ci] + [vp, i64, i64] * 8 + [i64, i64, i64, i64, ci, vp, sz, vp]
         L.pf_lowrank_conv_workspace.restype = sz
         L.pf_lowrank_conv_workspace.argtypes = [ci] * 12
         L.pf_lowrank_conv_fwd.restype = ci
@@ -206,6 +212,74 @@ def pf_lowrank_linear_bwd(x, U, V, dY, *, T_stash=None, need_dX=True, dX=None, d
         return _Prepared(lib().pf_lowrank_linear_bwd, args, "pf_lowrank_linear_bwd",
                          (x, U, V, dY, T_stash, dX, dU, dV, ws)), (dX, dU, dV)
     _check(lib().pf_lowrank_linear_bwd(*args), "pf_lowrank_linear_bwd")
+    return dX, dU, dV
+
+
+def pf_lowrank_linear_grouped_workspace(groups, m, k, n, r, dtype, is_bwd) -> int:
+    return int(lib().pf_lowrank_linear_grouped_workspace(groups, m, k, n, r, dtype, int(bool(is_bwd))))
+
+
+def _grp(t: torch.Tensor, name: str, groups: int, may_share: bool = False):
+    """(pointer, row pitch, group stride) of a [groups, rows, cols] tensor (unit column stride), or of
+    a 2-D [rows, cols] tensor shared by all groups (stride 0) where that is allowed."""
+    if t is None:
+        return ctypes.c_void_p(0), 0, 0
+    if t.dim() == 2 and may_share:
+        return _ptr(t), _mat(t, name), 0
+    if not t.is_cuda or t.dim() != 3 or t.shape[0] != groups or (t.shape[2] > 1 and t.stride(2) != 1):
+        raise ValueError(f"{name}: need a CUDA tensor [groups, rows, cols] with unit column stride")
+    ld = t.stride(1) if t.shape[1] > 1 else max(t.stride(1), t.shape[2])
+    return _ptr(t), ld, t.stride(0)
+
+
+def pf_lowrank_linear_grouped_fwd(x, U, V, *, y=None, T_stash=None, want_stash=False, workspace=None,
+                                  stream=None, prepare=False):
+    """y[g] = (x[g] U[g]) V[g]^T for U [G, k, r], V [G, n, r] and x [G, m, k] or one shared x [m, k].
+    Returns y [G, m, n], or (y, T_stash [G, m, r]) when a stash is requested."""
+    dt = _dtype_code(U)
+    G, k, r = U.shape
+    n = V.shape[1]
+    m = x.shape[-2]
+    if V.shape != (G, n, r) or x.shape[-1] != k:
+        raise ValueError("U must be [G, k, r], V [G, n, r], x [G, m, k] or [m, k]")
+    if y is None:
+        y = torch.empty((G, m, n), dtype=U.dtype, device=U.device)
+    if T_stash is None and want_stash:
+        T_stash = torch.empty((G, m, r), dtype=U.dtype, device=U.device)
+    ws = _workspace(pf_lowrank_linear_grouped_workspace(G, m, k, n, r, dt, 0), U.device, workspace, stream)
+    args = (G, *_grp(x, "x", G, True), *_grp(U, "U", G), *_grp(V, "V", G), *_grp(y, "y", G), *_grp(T_stash, "T_stash", G),
+            m, k, n, r, dt, _ptr(ws), ws.numel(), _stream(stream))
+    out = (y, T_stash) if T_stash is not None else y
+    if prepare:
+        return _Prepared(lib().pf_lowrank_linear_grouped_fwd, args, "pf_lowrank_linear_grouped_fwd",
+                         (x, U, V, y, T_stash, ws)), out
+    _check(lib().pf_lowrank_linear_grouped_fwd(*args), "pf_lowrank_linear_grouped_fwd")
+    return out
+
+
+def pf_lowrank_linear_grouped_bwd(x, U, V, dY, *, T_stash=None, need_dX=True, dX=None, dU=None, dV=None,
+                                  workspace=None, stream=None, prepare=False):
+    """Returns (dX or None, dU [G, k, r], dV [G, n, r]).  dX is [G, m, k] when every group has its own
+    x and ONE [m, k] matrix (the sum over the groups) when x [m, k] is shared."""
+    dt = _dtype_code(U)
+    G, k, r = U.shape
+    n = V.shape[1]
+    m = x.shape[-2]
+    shared = x.dim() == 2
+    if dX is None and need_dX:
+        dX = torch.empty((m, k) if shared else (G, m, k), dtype=U.dtype, device=U.device)
+    if dU is None:
+        dU = torch.empty_like(U)
+    if dV is None:
+        dV = torch.empty_like(V)
+    ws = _workspace(pf_lowrank_linear_grouped_workspace(G, m, k, n, r, dt, 1), U.device, workspace, stream)
+    args = (G, *_grp(x, "x", G, True), *_grp(U, "U", G), *_grp(V, "V", G), *_grp(dY, "dY", G), *_grp(T_stash, "T_stash", G),
+            *_grp(dX, "dX", G, True), *_grp(dU, "dU", G), *_grp(dV, "dV", G),
+            m, k, n, r, dt, _ptr(ws), ws.numel(), _stream(stream))
+    if prepare:
+        return _Prepared(lib().pf_lowrank_linear_grouped_bwd, args, "pf_lowrank_linear_grouped_bwd",
+                         (x, U, V, dY, T_stash, dX, dU, dV, ws)), (dX, dU, dV)
+    _check(lib().pf_lowrank_linear_grouped_bwd(*args), "pf_lowrank_linear_grouped_bwd")
     return dX, dU, dV
 
 

@@ -260,6 +260,132 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
     return PF_OK;
 }
 
+// ------------------------------------------------------------------------------ grouped linear
+namespace {
+struct GroupedWs {
+    size_t off_tc, off_acc, off_dx, off_single, total;
+};
+// Workspace of the grouped calls: the tensor-core path's buffers, then (for the path that runs group by
+// group) an fp32 accumulator and one per-group dX for layers whose groups share x, then the workspace
+// of one ungrouped call.
+GroupedWs grouped_ws(int groups, int64_t m, int64_t k, int64_t n, int64_t r, int dtype, bool bwd) {
+    GroupedWs w;
+    size_t off = 0;
+    w.off_tc = off;
+    if (dtype == PF_BF16) off += align_up(tc::grouped_workspace(groups, m, k, n, r, bwd), 256);
+    w.off_acc = off;
+    if (bwd) off += align_up(static_cast<size_t>(m) * k * 4, 256);
+    w.off_dx = off;
+    if (bwd) off += align_up(static_cast<size_t>(m) * k * dtype_size(dtype), 256);
+    w.off_single = off;
+    off += linear_ws(m, k, n, r, dtype, bwd).total;
+    w.total = off;
+    return w;
+}
+const void* at_c(const void* p, int64_t stride, int g, int dtype) {
+    return p ? static_cast<const char*>(p) + static_cast<size_t>(g) * stride * dtype_size(dtype) : nullptr;
+}
+void* at_m(void* p, int64_t stride, int g, int dtype) {
+    return p ? static_cast<char*>(p) + static_cast<size_t>(g) * stride * dtype_size(dtype) : nullptr;
+}
+}  // namespace
+
+size_t pf_lowrank_linear_grouped_workspace(int groups, int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                                           int is_bwd) {
+    if (!valid_dtype(dtype) || groups < 1 || m < 0 || k < 1 || n < 1 || r < 1) return 0;
+    return grouped_ws(groups, m, k, n, r, dtype, is_bwd != 0).total;
+}
+
+int pf_lowrank_linear_grouped_fwd(int groups, const void* x, int64_t ldx, int64_t sx, const void* U, int64_t ldu,
+                                  int64_t su, const void* V, int64_t ldv, int64_t sv, void* y, int64_t ldy, int64_t sy,
+                                  void* T_stash, int64_t ldt, int64_t st, int64_t m, int64_t k, int64_t n, int64_t r,
+                                  int dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (groups < 1 || sx < 0 || su < 0 || sv < 0 || sy < 0 || st < 0) return PF_ERR_INVALID_ARG;
+    int rc = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
+    if (rc != PF_OK) return rc;
+    if ((!y && m > 0) || ldy < n || !elem_aligned(y, dtype)) return PF_ERR_INVALID_ARG;
+    if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
+    // every group has its own factors and outputs; only x may be shared (sx == 0)
+    if (groups > 1 && (su < k * ldu - (ldu - r) || sv < n * ldv - (ldv - r) || (m > 0 && sy < (m - 1) * ldy + n) ||
+                       (T_stash && m > 0 && st < (m - 1) * ldt + r) || (sx != 0 && m > 0 && sx < (m - 1) * ldx + k)))
+        return PF_ERR_INVALID_ARG;
+    const GroupedWs w = grouped_ws(groups, m, k, n, r, dtype, false);
+    rc = check_ws(workspace, workspace_bytes, w.total);
+    if (rc != PF_OK) return rc;
+    if (m == 0) return PF_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    if (dtype == PF_BF16) {
+        tc::GroupedArgs a;
+        a.groups = groups; a.x = x; a.ldx = ldx; a.sx = sx; a.U = U; a.ldu = ldu; a.su = su; a.V = V; a.ldv = ldv; a.sv = sv;
+        a.y = y; a.ldy = ldy; a.sy = sy; a.T = T_stash; a.ldt = ldt; a.st = st;
+        a.m = m; a.k = k; a.n = n; a.r = r; a.ws = ws + w.off_tc; a.stream = stream;
+        int handled = 0;
+        rc = tc::linear_grouped_fwd(a, &handled);
+        if (rc != PF_OK || handled) return rc;
+    }
+    // group by group through the ungrouped entry (fp32, and bf16 operands TMA cannot describe)
+    const size_t single = linear_ws(m, k, n, r, dtype, false).total;
+    for (int g = 0; g < groups; ++g) {
+        rc = linear_fwd_impl(at_c(x, sx, g, dtype), ldx, at_c(U, su, g, dtype), ldu, at_c(V, sv, g, dtype), ldv, at_m(y, sy, g, dtype),
+                             ldy, at_m(T_stash, st, g, dtype), ldt, m, k, n, r, dtype, ws + w.off_single, single, cuda_stream,
+                             false);
+        if (rc != PF_OK) return rc;
+    }
+    return PF_OK;
+}
+
+int pf_lowrank_linear_grouped_bwd(int groups, const void* x, int64_t ldx, int64_t sx, const void* U, int64_t ldu,
+                                  int64_t su, const void* V, int64_t ldv, int64_t sv, const void* dY, int64_t lddy,
+                                  int64_t sdy, const void* T_stash, int64_t ldt, int64_t st, void* dX, int64_t lddx,
+                                  int64_t sdx, void* dU, int64_t lddu, int64_t sdu, void* dV, int64_t lddv, int64_t sdv,
+                                  int64_t m, int64_t k, int64_t n, int64_t r, int dtype, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
+    if (groups < 1 || sx < 0 || su < 0 || sv < 0 || sdy < 0 || st < 0 || sdx < 0 || sdu < 0 || sdv < 0) return PF_ERR_INVALID_ARG;
+    int rc = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
+    if (rc != PF_OK) return rc;
+    if ((!dY && m > 0) || lddy < n || !elem_aligned(dY, dtype)) return PF_ERR_INVALID_ARG;
+    if (!dU || lddu < r || !elem_aligned(dU, dtype) || !dV || lddv < r || !elem_aligned(dV, dtype)) return PF_ERR_INVALID_ARG;
+    if (dX && (lddx < k || !elem_aligned(dX, dtype))) return PF_ERR_INVALID_ARG;
+    if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
+    const bool shared_x = sx == 0 && groups > 1;
+    if (groups > 1 && (su < k * ldu - (ldu - r) || sv < n * ldv - (ldv - r) || sdu < k * lddu - (lddu - r) ||
+                       sdv < n * lddv - (lddv - r) || (m > 0 && sdy < (m - 1) * lddy + n) ||
+                       (T_stash && m > 0 && st < (m - 1) * ldt + r) || (sx != 0 && m > 0 && sx < (m - 1) * ldx + k) ||
+                       (dX && !shared_x && m > 0 && sdx < (m - 1) * lddx + k)))
+        return PF_ERR_INVALID_ARG;
+    const GroupedWs w = grouped_ws(groups, m, k, n, r, dtype, true);
+    rc = check_ws(workspace, workspace_bytes, w.total);
+    if (rc != PF_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    if (dtype == PF_BF16 && m > 0) {
+        tc::GroupedArgs a;
+        a.groups = groups; a.x = x; a.ldx = ldx; a.sx = sx; a.U = U; a.ldu = ldu; a.su = su; a.V = V; a.ldv = ldv; a.sv = sv;
+        a.dY = dY; a.lddy = lddy; a.sdy = sdy; a.T = const_cast<void*>(T_stash); a.ldt = ldt; a.st = st;
+        a.dX = dX; a.lddx = lddx; a.sdx = sdx; a.dU = dU; a.lddu = lddu; a.sdu = sdu; a.dV = dV; a.lddv = lddv; a.sdv = sdv;
+        a.m = m; a.k = k; a.n = n; a.r = r; a.ws = ws + w.off_tc; a.stream = stream;
+        int handled = 0;
+        rc = tc::linear_grouped_bwd(a, &handled);
+        if (rc != PF_OK || handled) return rc;
+    }
+    // group by group; groups that share x add their input gradients in an fp32 accumulator
+    const size_t single = linear_ws(m, k, n, r, dtype, true).total;
+    float* acc = reinterpret_cast<float*>(ws + w.off_acc);
+    void* dx_one = ws + w.off_dx;
+    for (int g = 0; g < groups; ++g) {
+        void* dx_g = !dX ? nullptr : shared_x ? dx_one : at_m(dX, sdx, g, dtype);
+        rc = pf_lowrank_linear_bwd(at_c(x, sx, g, dtype), ldx, at_c(U, su, g, dtype), ldu, at_c(V, sv, g, dtype), ldv,
+                                   at_c(dY, sdy, g, dtype), lddy, at_c(T_stash, st, g, dtype), ldt, dx_g, shared_x ? k : lddx,
+                                   at_m(dU, sdu, g, dtype), lddu, at_m(dV, sdv, g, dtype), lddv, m, k, n, r, dtype,
+                                   ws + w.off_single, single, cuda_stream);
+        if (rc != PF_OK) return rc;
+        if (dX && shared_x && m > 0) PF_CUDA(accumulate_f32(acc, dx_one, k, m, k, dtype, g == 0, stream));
+    }
+    if (dX && shared_x && m > 0) PF_CUDA(round_out_f32(acc, dX, lddx, m, k, dtype, stream));
+    return PF_OK;
+}
+
 // ------------------------------------------------------------------------------ conv
 namespace {
 struct ConvWs {

@@ -85,6 +85,12 @@ cudaError_t splitk_reduce(const float* partial, void* C, int64_t ldc, int64_t M,
 cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t ld_dst,
                              int64_t rows, int64_t cols, int64_t cols_padded, cudaStream_t stream);
 
+// acc (fp32, dense [rows, cols]) = (first ? 0 : acc) + src; dst = acc rounded once to the storage dtype.
+cudaError_t accumulate_f32(float* acc, const void* src, int64_t ld_src, int64_t rows, int64_t cols, int dtype, bool first,
+                           cudaStream_t stream);
+cudaError_t round_out_f32(const float* acc, void* dst, int64_t ld_dst, int64_t rows, int64_t cols, int dtype,
+                          cudaStream_t stream);
+
 // Several such copies in one launch (row counts and widths below 2^31).
 struct RepackJob {
     const void* src;

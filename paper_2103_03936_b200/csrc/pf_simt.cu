@@ -256,6 +256,53 @@ cudaError_t simt_gemm(const SimtGemm& g, cudaStream_t stream) {
     return g.dtype == PF_BF16 ? launch_typed<__nv_bfloat16>(g, stream) : launch_typed<float>(g, stream);
 }
 
+// acc[rows, cols] (fp32, dense) = (first ? 0 : acc) + src (storage dtype, pitch ld_src); and its
+// counterpart that rounds the sums to the storage dtype once.  They add up the per-group input
+// gradients of a grouped layer whose groups share one input, on the path that runs group by group.
+template <typename T>
+__global__ void accumulate_kernel(float* acc, const T* src, int64_t ld_src, int64_t rows, int64_t cols, int first) {
+    const int64_t total = rows * cols;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t rr = i / cols, cc = i - rr * cols;
+        const float v = static_cast<float>(src[rr * ld_src + cc]);
+        acc[i] = first ? v : acc[i] + v;
+    }
+}
+template <typename T>
+__global__ void round_out_kernel(const float* acc, T* dst, int64_t ld_dst, int64_t rows, int64_t cols) {
+    const int64_t total = rows * cols;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t rr = i / cols, cc = i - rr * cols;
+        dst[rr * ld_dst + cc] = static_cast<T>(acc[i]);
+    }
+}
+cudaError_t accumulate_f32(float* acc, const void* src, int64_t ld_src, int64_t rows, int64_t cols, int dtype, bool first,
+                           cudaStream_t stream) {
+    const int64_t total = rows * cols;
+    if (total <= 0) return cudaSuccess;
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 8 * num_sms() ? ceil_div(total, 256) : 8 * num_sms());
+    if (dtype == PF_BF16)
+        accumulate_kernel<<<blocks, 256, 0, stream>>>(acc, static_cast<const __nv_bfloat16*>(src), ld_src, rows, cols, first ? 1 : 0);
+    else
+        accumulate_kernel<<<blocks, 256, 0, stream>>>(acc, static_cast<const float*>(src), ld_src, rows, cols, first ? 1 : 0);
+    count_launch();
+    return cudaGetLastError();
+}
+cudaError_t round_out_f32(const float* acc, void* dst, int64_t ld_dst, int64_t rows, int64_t cols, int dtype,
+                          cudaStream_t stream) {
+    const int64_t total = rows * cols;
+    if (total <= 0) return cudaSuccess;
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 8 * num_sms() ? ceil_div(total, 256) : 8 * num_sms());
+    if (dtype == PF_BF16)
+        round_out_kernel<<<blocks, 256, 0, stream>>>(acc, static_cast<__nv_bfloat16*>(dst), ld_dst, rows, cols);
+    else
+        round_out_kernel<<<blocks, 256, 0, stream>>>(acc, static_cast<float*>(dst), ld_dst, rows, cols);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t repack_rows_bf16(const void* src, int64_t ld_src, void* dst, int64_t ld_dst,
                              int64_t rows, int64_t cols, int64_t cols_padded, cudaStream_t stream) {
     const int64_t total = rows * cols_padded;

@@ -14,6 +14,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <mutex>
 
 #include "pf_tc_host.h"
 #include "pf_tc_prims.cuh"
@@ -68,12 +69,26 @@ struct GemmParams {
     int kpix;                // conv_mode 2: pixels per k-block (cv_box_h * W <= 64), else 64
     int nkb_total;           // k-blocks of the whole contraction
     int independent;         // 1: reads nothing the preceding kernel of the stream writes (see gemm_tile)
+    // Grouped products (several problems of one shape in a launch): tmA / tmB are 3-D maps whose outermost
+    // coordinate is the group (a shared operand has one group only), outputs of group g start g * c_gstride
+    // elements after C.  kb_per_group > 0 instead makes the group part of the CONTRACTION: k-block kb reads
+    // group kb / kb_per_group, 64-element block kb % kb_per_group of both operands (the sum over groups of
+    // A_g B_g^T, i.e. dX of several factor pairs that share one input).
+    int groups, a_shared, b_shared, kb_per_group, tiles_y;
+    long long c_gstride;
 };
 
 __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
     unsigned int v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
 }
 
 // One output tile (128 rows x BN columns) of C = A * B, or one slice of its contraction.
@@ -86,7 +101,7 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
 // order, its share of the rows over all slices and writes bf16 (bit-reproducible, no second launch).
 template <int BN>
 __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
-                                          const int bx, const int by, const int bz) {
+                                          const int bx, const int by, const int bz, const int bg) {
     constexpr uint32_t kABytes = kBM * kBK * 2;          // 16 KB
     constexpr uint32_t kBBytes = BN * kBK * 2;
     constexpr uint32_t kStageBytes = kABytes + kBBytes;
@@ -104,7 +119,8 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     const int kb_end = min(nkb_total, kb_beg + p.kb_per_split);
     const int nkb = kb_end - kb_beg;
     const uint32_t NS = static_cast<uint32_t>(p.num_stages);
-    const int tile = by * p.tiles_x + bx;
+    const int tile = (bg * p.tiles_y + by) * p.tiles_x + bx;
+    const bool grouped = p.groups > 1 || p.kb_per_group > 0;
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < NS; ++s) {
@@ -133,13 +149,9 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    // A product marked independent reads nothing that the kernel launched just before it writes, so
-    // it does not wait for that kernel: its blocks run beside it on SMs that kernel leaves free.  (Every
-    // kernel of this library lets its successor start only after its own wait has returned, i.e. once
-    // everything older in the stream is complete, so older results are safe to read.)
     // While the previous kernel of the stream finishes, ask L2 for this block's first tiles (a prefetch
     // only moves lines into L2, the point of coherence: harmless even if that kernel still writes them).
-    if (p.conv_mode == 0 && (warp == 0 || warp == 6) && elect_one()) {
+    if (p.conv_mode == 0 && !grouped && (warp == 0 || warp == 6) && elect_one()) {
         for (int i = 0; i < 6 && i < nkb; ++i) {
             const int k0 = (kb_beg + i) * kBK;
             if (warp == 0) {
@@ -153,6 +165,10 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
             }
         }
     }
+    // A product marked independent reads nothing that the kernel launched just before it writes, so
+    // it does not wait for that kernel: its blocks run beside it on SMs that kernel leaves free.  (Every
+    // kernel of this library lets its successor start only after its own wait has returned, i.e. once
+    // everything older in the stream is complete, so older results are safe to read.)
     if (!p.independent) pdl_wait();     // everything above overlapped the previous kernel's tail
     pdl_launch_dependents();
     const uint32_t tmem_base = ctl->tmem_base;
@@ -220,6 +236,29 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
                     if (++c2_t == p.cv_tpi) { c2_t = 0; ++c2_img; }
                     if (++s == NS) { s = 0; ph ^= 1u; }
                     continue;
+                } else if (grouped) {
+                    int g = bg, kk0 = k0;
+                    if (p.kb_per_group > 0) {
+                        g = (kb_beg + i) / p.kb_per_group;
+                        kk0 = ((kb_beg + i) - g * p.kb_per_group) * kBK;
+                    }
+                    if (do_a) {
+                        const int ga = p.a_shared ? 0 : g;
+                        if (p.a_mn) {
+                            tma_load_3d(a_dst, &tmA, full, m0, kk0, ga);
+                            tma_load_3d(a_dst + 8192, &tmA, full, m0 + 64, kk0, ga);
+                        } else {
+                            tma_load_3d(a_dst, &tmA, full, kk0, m0, ga);
+                        }
+                    } else {
+                        const int gb = p.b_shared ? 0 : g;
+                        if (p.b_mn) {
+#pragma unroll
+                            for (int h = 0; h < BN / 64; ++h) tma_load_3d(b_dst + h * 8192, &tmB, full, n0 + 64 * h, kk0, gb);
+                        } else {
+                            tma_load_3d(b_dst, &tmB, full, kk0, n0, gb);
+                        }
+                    }
                 } else if (do_a) {
                     if (p.a_mn) {
                         tma_load_2d(a_dst, &tmA, full, m0, k0);
@@ -304,9 +343,9 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
             } else {
                 // every MMA has completed, so the pipeline stages are free: 32 x 33-word panel per warp
                 uint32_t* stg = reinterpret_cast<uint32_t*>(tiles) + (warp - 2) * (32 * 33);
-                __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
-                const bool pair_ok = (p.ldc % 2) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 3) == 0;
-                const bool vec_ok = (p.ldc % 8) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 15) == 0;
+                __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C) + static_cast<long long>(bg) * p.c_gstride;
+                const bool pair_ok = (p.ldc % 2) == 0 && (reinterpret_cast<uintptr_t>(Cb) & 3) == 0;
+                const bool vec_ok = (p.ldc % 8) == 0 && (reinterpret_cast<uintptr_t>(Cb) & 15) == 0;
                 if (vec_ok) {
                     // 16-byte aligned rows: stage 32 rows x 64 columns (128 bytes per row, 16-byte pieces
                     // XOR-swizzled by the row so that both passes are free of bank conflicts), then
@@ -439,10 +478,10 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     }
     __syncthreads();
     if (ctl->fix_ok) {
-        __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
+        __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C) + static_cast<long long>(bg) * p.c_gstride;
         __nv_bfloat16* C2b = reinterpret_cast<__nv_bfloat16*>(p.C2);
         const uint32_t base = smem_u32(tiles);
-        const bool vec8 = (p.ldc % 4) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 7) == 0;
+        const bool vec8 = (p.ldc % 4) == 0 && (reinterpret_cast<uintptr_t>(Cb) & 7) == 0;
         // consecutive threads take consecutive 16-byte pieces of one row
         for (int id = threadIdx.x; id < nr * static_cast<int>(kPieces); id += kGemmThreads) {
             const int rl = id / static_cast<int>(kPieces), pc = id % static_cast<int>(kPieces);
@@ -493,7 +532,8 @@ template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, BN <= 128 ? 2 : 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const GemmParams p) {
-    gemm_tile<BN>(tmA, tmB, p, blockIdx.x, blockIdx.y, blockIdx.z);
+    const int sl = p.splits < 1 ? 1 : p.splits;
+    gemm_tile<BN>(tmA, tmB, p, blockIdx.x, blockIdx.y, static_cast<int>(blockIdx.z) % sl, static_cast<int>(blockIdx.z) / sl);
 }
 
 // Up to three independent products in one launch (dU = x^T G, dV = dY^T T and, where it is a plain
@@ -503,9 +543,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // Tiles may be 64 or 128 columns wide per product.
 __device__ __forceinline__ void gemm_any(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int idx,
                                          const int2 t) {
-    const int bx = idx % t.x, by = (idx / t.x) % t.y, bz = idx / (t.x * t.y);
-    if (p.bn == 64) gemm_tile<64>(tmA, tmB, p, bx, by, bz);
-    else gemm_tile<128>(tmA, tmB, p, bx, by, bz);
+    const int sl = p.splits < 1 ? 1 : p.splits;
+    const int bx = idx % t.x, by = (idx / t.x) % t.y, zz = idx / (t.x * t.y);
+    if (p.bn == 64) gemm_tile<64>(tmA, tmB, p, bx, by, zz % sl, zz / sl);
+    else gemm_tile<128>(tmA, tmB, p, bx, by, zz % sl, zz / sl);
 }
 __global__ void __launch_bounds__(kGemmThreads, 2)
 tc_gemm3_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
@@ -526,7 +567,55 @@ struct Operand {
     const void* p;
     int64_t ld;
     bool mn_major;
+    int64_t gs = 0;     // grouped products: elements between the matrices of consecutive groups (0 = one matrix shared by all)
 };
+
+// Several problems of one shape in one product.  sum_groups: the groups are summed into ONE output (the
+// group index is part of the contraction; both operands K-major), otherwise every group has its own
+// output, c_gs elements apart.
+struct Grouping {
+    int groups = 1;
+    int64_t c_gs = 0;
+    bool sum_groups = false;
+};
+
+// 3-D bf16 tensor map over `groups` row-major [rows, cols] matrices gs elements apart (boxes of 64 columns x
+// box_rows rows of one group; out-of-range elements read as zero).  Cached like the 2-D maps.
+bool cached_map_3d(CUtensorMap* map, const void* p, int64_t groups, int64_t rows, int64_t cols, int64_t ld, int64_t gs,
+                   int box_rows) {
+    constexpr int kSlots = 128;
+    struct Key { const void* p; int64_t groups, rows, cols, ld, gs; int box_rows; };
+    struct Slot { Key key; CUtensorMap map; bool used; };
+    static Slot slots[kSlots];
+    static std::mutex mu;
+    if (groups < 1) return false;
+    if (groups == 1) gs = rows * ld;                       // a single group: any valid stride
+    if ((gs * 2) % 16 != 0 || gs * 2 >= (1LL << 40)) return false;
+    uint64_t h = reinterpret_cast<uintptr_t>(p) * 0x9E3779B97F4A7C15ull;
+    h ^= static_cast<uint64_t>(rows) * 0xC2B2AE3D27D4EB4Full + static_cast<uint64_t>(cols) * 0x165667B19E3779F9ull +
+         static_cast<uint64_t>(ld) * 31 + static_cast<uint64_t>(box_rows) + static_cast<uint64_t>(gs) * 131 + static_cast<uint64_t>(groups) * 7;
+    Slot& sl = slots[(h >> 20) % kSlots];
+    std::lock_guard<std::mutex> lock(mu);
+    const Key& k = sl.key;
+    if (sl.used && k.p == p && k.groups == groups && k.rows == rows && k.cols == cols && k.ld == ld && k.gs == gs &&
+        k.box_rows == box_rows) {
+        *map = sl.map;
+        return true;
+    }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(groups)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld) * 2, static_cast<cuuint64_t>(gs) * 2};
+    const cuuint32_t box[3] = {64u, static_cast<cuuint32_t>(box_rows), 1u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(p), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    sl.key = Key{p, groups, rows, cols, ld, gs, box_rows};
+    sl.map = *map;
+    sl.used = true;
+    return true;
+}
 
 size_t gemm_smem(int bn, int stages) {
     return 1024 + 1024 + static_cast<size_t>(stages) * (kBM * kBK * 2 + bn * kBK * 2);
@@ -671,8 +760,11 @@ struct GemmLaunch {
 
 // Encodes the tensor maps and launch geometry of C[M,N] = A * B without launching.
 int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
-                 int splits, float* partial, const ConvA* cv, GemmLaunch* out) {
+                 int splits, float* partial, const ConvA* cv, GemmLaunch* out, const Grouping* gr = nullptr) {
     if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PF_ERR_UNSUPPORTED;
+    const int groups = gr ? gr->groups : 1;
+    const bool sum_groups = gr && gr->sum_groups;
+    if (gr && (cv || groups < 1 || groups > 1024 || (sum_groups && (A.mn_major || B.mn_major)))) return PF_ERR_UNSUPPORTED;
     // wide outputs that would need more than one wave of 128-column tiles (two CTAs per SM) take
     // 256-column tiles
     const int bn = (splits <= 1 && N >= 512 && ceil_div(M, kBM) * ceil_div(N, 128) > 2 * num_sms()) ? 256 : pick_bn(N);
@@ -685,6 +777,10 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     } else if (cv && cv->mode == 2) {
         oka = cached_map_nhwc(&ta, A.p, cv->N, cv->H, cv->W, cv->Cimg, cv->W, conv_box_h(cv->H, cv->W, 64));
         okb = cached_map_2d(&tb, B.p, K, N, B.ld, 64);
+    } else if (gr) {
+        const int64_t ga = A.gs == 0 ? 1 : groups, gb = B.gs == 0 ? 1 : groups;
+        oka = A.mn_major ? cached_map_3d(&ta, A.p, ga, K, M, A.ld, A.gs, 64) : cached_map_3d(&ta, A.p, ga, M, K, A.ld, A.gs, kBM);
+        okb = B.mn_major ? cached_map_3d(&tb, B.p, gb, K, N, B.ld, B.gs, 64) : cached_map_3d(&tb, B.p, gb, N, K, B.ld, B.gs, bn);
     } else {
         oka = A.mn_major ? cached_map_2d(&ta, A.p, K, M, A.ld, 64) : cached_map_2d(&ta, A.p, M, K, A.ld, kBM);
         okb = B.mn_major ? cached_map_2d(&tb, B.p, K, N, B.ld, 64) : cached_map_2d(&tb, B.p, N, K, B.ld, bn);
@@ -704,22 +800,33 @@ int gemm_prepare(const Operand& A, const Operand& B, int64_t M, int64_t N, int64
     }
     p.rows_tile = (cv && cv->mode == 1) ? p.cv_box_h * cv->W : kBM;
     p.kpix = (cv && cv->mode == 2) ? p.cv_box_h * cv->W : kBK;
-    const int64_t nkb = ceil_div(K, p.kpix);
+    p.groups = gr ? groups : 1;
+    p.a_shared = gr && A.gs == 0; p.b_shared = gr && B.gs == 0;
+    p.c_gstride = gr ? gr->c_gs : 0;
+    p.kb_per_group = 0;
+    int64_t nkb = ceil_div(K, p.kpix);
+    if (sum_groups) {                       // the groups are part of the contraction: one output
+        p.kb_per_group = static_cast<int>(nkb);
+        nkb *= groups;
+        p.groups = 1;
+    }
+    const int out_groups = sum_groups ? 1 : groups;
     p.nkb_total = static_cast<int>(nkb);
     p.kb_per_split = static_cast<int>(ceil_div(nkb, splits < 1 ? 1 : splits));
     p.splits = static_cast<int>(ceil_div(nkb, p.kb_per_split));   // every slice gets >= 1 k-block
     p.status = device_status_ptr();
     dim3 grid(static_cast<unsigned>(ceil_div(M, p.rows_tile)), static_cast<unsigned>(ceil_div(N, bn)),
-              static_cast<unsigned>(p.splits));
-    if (grid.y > 65535) return PF_ERR_UNSUPPORTED;
+              static_cast<unsigned>(p.splits * out_groups));
+    if (grid.y > 65535 || grid.z > 65535) return PF_ERR_UNSUPPORTED;
     p.tiles_x = static_cast<int>(grid.x);
+    p.tiles_y = static_cast<int>(grid.y);
     p.bn = bn;
     p.num_stages = pick_stages(bn, static_cast<int64_t>(grid.x) * grid.y * grid.z);
     p.counters = nullptr;
     p.independent = 0;
     if (p.splits > 1) {
         // the CTAs of a tile wait for one another, so all of them must be resident at once
-        if (static_cast<int64_t>(grid.x) * grid.y > kFixTiles || static_cast<int64_t>(grid.x) * grid.y * grid.z > num_sms() ||
+        if (static_cast<int64_t>(grid.x) * grid.y * out_groups > kFixTiles || static_cast<int64_t>(grid.x) * grid.y * grid.z > num_sms() ||
             bn == 256 || partial == nullptr)
             return PF_ERR_UNSUPPORTED;
         // the slices of a CTA's share are gathered in the pipeline stages
@@ -1104,6 +1211,118 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream);
     if (st != PF_OK) return st;
     return gemm({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, a.stream);
+}
+
+// ------------------------------------------------------------------------------ grouped linear layer
+namespace {
+int grouped_splits(int64_t tiles, int64_t nkb) {
+    int64_t s = num_sms() / std::max<int64_t>(tiles, 1);
+    s = std::min<int64_t>(s, std::min<int64_t>(64, nkb / 4));
+    return static_cast<int>(std::max<int64_t>(s, 1));
+}
+struct GroupedPlan {
+    int bn;                       // tile width of the m x r and (k|n) x r products
+    int s1, sg, su, sv;           // slices of x U, dY V, dU, dV
+    size_t t_bytes, p1_bytes, pu_bytes, pv_bytes;
+};
+GroupedPlan grouped_plan(int groups, int64_t m, int64_t k, int64_t n, int64_t r) {
+    GroupedPlan g;
+    g.bn = pick_bn(r);
+    const int64_t tr = ceil_div(r, g.bn);
+    const int64_t tm = ceil_div(m, kBM) * tr * groups, tk = ceil_div(k, kBM) * tr * groups, tn = ceil_div(n, kBM) * tr * groups;
+    g.s1 = grouped_splits(tm, ceil_div(k, kBK));
+    g.sg = grouped_splits(tm, ceil_div(n, kBK));
+    g.su = grouped_splits(tk, ceil_div(m, kBK));
+    g.sv = grouped_splits(tn, ceil_div(m, kBK));
+    if (tm > kFixTiles) g.s1 = g.sg = 1;
+    if (tk > kFixTiles) g.su = 1;
+    if (tn > kFixTiles) g.sv = 1;
+    g.t_bytes = align_up(static_cast<size_t>(groups) * m * pad8(r) * 2, 256);
+    g.p1_bytes = align_up(static_cast<size_t>(groups) * std::max(partial_bytes(m, r, g.s1), partial_bytes(m, r, g.sg)), 256);
+    g.pu_bytes = align_up(static_cast<size_t>(groups) * partial_bytes(k, r, g.su), 256);
+    g.pv_bytes = align_up(static_cast<size_t>(groups) * partial_bytes(n, r, g.sv), 256);
+    return g;
+}
+bool grouped_ok(const void* p, int64_t ld, int64_t gs) { return tma_ok(p, ld) && gs % 8 == 0; }
+}  // namespace
+
+size_t grouped_workspace(int groups, int64_t m, int64_t k, int64_t n, int64_t r, bool bwd) {
+    const GroupedPlan g = grouped_plan(groups, m, k, n, r);
+    return g.t_bytes + g.p1_bytes + (bwd ? g.t_bytes + g.pu_bytes + g.pv_bytes : 0);
+}
+
+int linear_grouped_fwd(const GroupedArgs& a, int* handled) {
+    *handled = 0;
+    if (encode_fn() == nullptr || a.groups > 1024 || a.k > (1 << 22) || a.n > (1 << 22) || a.r > (1 << 22)) return PF_OK;
+    if (!grouped_ok(a.x, a.ldx, a.sx) || !grouped_ok(a.U, a.ldu, a.su) || !grouped_ok(a.V, a.ldv, a.sv)) return PF_OK;
+    const GroupedPlan gp = grouped_plan(a.groups, a.m, a.k, a.n, a.r);
+    // T: the stash itself when TMA can read it back, else scratch at a padded pitch (copied out afterwards)
+    const bool stash_direct = a.T && grouped_ok(a.T, a.ldt, a.st);
+    if (a.T && !stash_direct) return PF_OK;
+    void* T = stash_direct ? a.T : static_cast<void*>(a.ws);
+    const int64_t ldT = stash_direct ? a.ldt : pad8(a.r), sT = stash_direct ? a.st : a.m * pad8(a.r);
+    float* p1 = reinterpret_cast<float*>(a.ws + gp.t_bytes);
+    GemmLaunch g1, g2;
+    const Grouping gt{a.groups, sT, false}, gy{a.groups, a.sy, false};
+    int st = gemm_prepare({a.x, a.ldx, false, a.sx}, {a.U, a.ldu, true, a.su}, a.m, a.r, a.k, T, ldT, gp.s1, p1, nullptr, &g1, &gt);
+    if (st == PF_OK)
+        st = gemm_prepare({T, ldT, false, sT}, {a.V, a.ldv, false, a.sv}, a.m, a.n, a.r, a.y, a.ldy, 1, nullptr, nullptr, &g2, &gy);
+    if (st == PF_ERR_UNSUPPORTED) return PF_OK;
+    if (st != PF_OK) return st;
+    *handled = 1;
+    st = launch_prepared(g1, a.stream);
+    if (st != PF_OK) return st;
+    return launch_prepared(g2, a.stream);
+}
+
+int linear_grouped_bwd(const GroupedArgs& a, int* handled) {
+    *handled = 0;
+    if (encode_fn() == nullptr || a.groups > 1024 || a.k > (1 << 22) || a.n > (1 << 22) || a.r > (1 << 22)) return PF_OK;
+    if (!grouped_ok(a.x, a.ldx, a.sx) || !grouped_ok(a.U, a.ldu, a.su) || !grouped_ok(a.V, a.ldv, a.sv) ||
+        !grouped_ok(a.dY, a.lddy, a.sdy) || (a.T && !grouped_ok(a.T, a.ldt, a.st)))
+        return PF_OK;
+    const GroupedPlan gp = grouped_plan(a.groups, a.m, a.k, a.n, a.r);
+    char* ws = a.ws;
+    void* Tbuf = ws; ws += gp.t_bytes;
+    float* p1 = reinterpret_cast<float*>(ws); ws += gp.p1_bytes;
+    void* Gbuf = ws; ws += gp.t_bytes;
+    float* pu = reinterpret_cast<float*>(ws); ws += gp.pu_bytes;
+    float* pv = reinterpret_cast<float*>(ws);
+    const int64_t ldW = pad8(a.r), sW = a.m * pad8(a.r);
+    const void* T = a.T ? a.T : Tbuf;
+    const int64_t ldT = a.T ? a.ldt : ldW, sT = a.T ? a.st : sW;
+    const bool shared_x = a.sx == 0 && a.groups > 1;
+    GemmLaunch gT, gG, gV, gU, gX;
+    const Grouping gw{a.groups, sW, false}, gdv{a.groups, a.sdv, false}, gdu{a.groups, a.sdu, false};
+    const Grouping gdx{a.groups, shared_x ? 0 : a.sdx, shared_x};
+    int st = PF_OK;
+    if (!a.T) st = gemm_prepare({a.x, a.ldx, false, a.sx}, {a.U, a.ldu, true, a.su}, a.m, a.r, a.k, Tbuf, ldW, gp.s1, p1, nullptr, &gT, &gw);
+    // the recomputed T and G share the slice buffer p1: they are separate launches, one after the other
+    if (st == PF_OK) st = gemm_prepare({a.dY, a.lddy, false, a.sdy}, {a.V, a.ldv, true, a.sv}, a.m, a.r, a.n, Gbuf, ldW, gp.sg, p1, nullptr, &gG, &gw);
+    if (st == PF_OK) st = gemm_prepare({a.dY, a.lddy, true, a.sdy}, {T, ldT, true, sT}, a.n, a.r, a.m, a.dV, a.lddv, gp.sv, pv, nullptr, &gV, &gdv);
+    if (st == PF_OK) st = gemm_prepare({a.x, a.ldx, true, a.sx}, {Gbuf, ldW, true, sW}, a.k, a.r, a.m, a.dU, a.lddu, gp.su, pu, nullptr, &gU, &gdu);
+    if (st == PF_OK && a.dX)
+        st = gemm_prepare({Gbuf, ldW, false, sW}, {a.U, a.ldu, false, a.su}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, nullptr, &gX, &gdx);
+    if (st == PF_ERR_UNSUPPORTED) return PF_OK;
+    if (st != PF_OK) return st;
+    *handled = 1;
+    if (!a.T) {
+        st = launch_prepared(gT, a.stream);
+        if (st != PF_OK) return st;
+    }
+    // launch A: G = dY V and dV = dY^T T (independent of each other); launch B: dU = x^T G and dX = G U^T
+    auto pair = [&](const GemmLaunch& p0, const GemmLaunch& q0, bool has_q) {
+        const GemmLaunch* list[2] = {&p0, &q0};
+        if (has_q && p0.p.splits <= 1 && q0.p.splits > 1) { list[0] = &q0; list[1] = &p0; }   // split products first
+        int r2 = gemm_multi(list, has_q ? 2 : 1, a.stream);
+        if (r2 != PF_ERR_UNSUPPORTED) return r2;
+        r2 = launch_prepared(p0, a.stream);
+        if (r2 == PF_OK && has_q) r2 = launch_prepared(q0, a.stream);
+        return r2;
+    };
+    st = pair(gG, gV, true);
+    if (st != PF_OK) return st;
+    return pair(gU, gX, a.dX != nullptr);
 }
 
 // After a bounded wait has expired some CTAs may have left their tile counters non-zero.

@@ -52,6 +52,24 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
 int gemm_pair_2sm(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb, bool b_mn, int64_t M, int64_t N,
                   int64_t K, void* C, int64_t ldc, cudaStream_t stream);
 
+// Grouped factorized linear layer: `groups` problems of one shape (several factor pairs applied to the
+// same or to different inputs) in two launches forward and two backward, whatever the group count.
+// Strides s* are in elements between consecutive groups; sx == 0 means one x shared by all groups,
+// in which case dX is ONE matrix, the sum over the groups.
+struct GroupedArgs {
+    int groups = 1;
+    const void *x = nullptr, *U = nullptr, *V = nullptr, *dY = nullptr;
+    void *y = nullptr, *T = nullptr, *dX = nullptr, *dU = nullptr, *dV = nullptr;
+    int64_t ldx = 0, ldu = 0, ldv = 0, ldy = 0, ldt = 0, lddy = 0, lddx = 0, lddu = 0, lddv = 0;
+    int64_t sx = 0, su = 0, sv = 0, sy = 0, st = 0, sdy = 0, sdx = 0, sdu = 0, sdv = 0;
+    int64_t m = 0, k = 0, n = 0, r = 0;
+    char* ws = nullptr;
+    cudaStream_t stream = nullptr;
+};
+size_t grouped_workspace(int groups, int64_t m, int64_t k, int64_t n, int64_t r, bool bwd);
+int linear_grouped_fwd(const GroupedArgs& a, int* handled);
+int linear_grouped_bwd(const GroupedArgs& a, int* handled);
+
 size_t linear_extra_workspace(int64_t m, int64_t k, int64_t n, int64_t r, bool bwd);
 size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
                             int pad, bool bwd);

@@ -133,3 +133,52 @@ def test_widen_returns_c_contiguous_for_sliced_bit_patterns():
     w = oracle.widen(U[..., [0, 2]])
     assert w.flags["C_CONTIGUOUS"]
     np.testing.assert_array_equal(w, np.arange(24.0).reshape(2, 3, 4)[..., [0, 2]])
+
+
+# ---------------------------------------------------------------------------------------------
+# grouped layer (per-gate LSTM factors of Section 2.3, attention projections of Section 2.4)
+def test_grouped_shared_input_equals_one_dense_layer_with_concatenated_weights():
+    """G factor pairs reading one x are the dense layer x [W_1 | ... | W_G] with W_g = U_g V_g^T
+    (the way the four gates of an LSTM are usually stored): outputs are its column blocks, and the
+    input gradient is dY_cat W_cat^T, i.e. the SUM over the groups.  Integers: exact."""
+    G, m, k, n, r = 3, 5, 4, 6, 2
+    x = rng_int(1, (m, k)); U = rng_int(2, (G, k, r)); V = rng_int(3, (G, n, r)); dY = rng_int(4, (G, m, n))
+    y, T = oracle.linear_grouped_fwd(x, U, V)
+    W_cat = np.concatenate([U[g] @ V[g].T for g in range(G)], axis=1)          # k x (G n)
+    np.testing.assert_array_equal(np.concatenate(list(y), axis=1), x @ W_cat)
+    np.testing.assert_array_equal(T, np.stack([x @ U[g] for g in range(G)]))
+    dX, dU, dV = oracle.linear_grouped_bwd(x, U, V, dY)
+    dY_cat = np.concatenate(list(dY), axis=1)
+    np.testing.assert_array_equal(dX, dY_cat @ W_cat.T)
+    dW_cat = x.T @ dY_cat                                                        # dense weight gradient
+    for g in range(G):
+        dW = dW_cat[:, g * n:(g + 1) * n]
+        np.testing.assert_array_equal(dU[g], dW @ V[g])
+        np.testing.assert_array_equal(dV[g], dW.T @ U[g])
+
+
+def test_grouped_own_inputs_is_a_block_diagonal_layer():
+    """Groups with their own x are one layer on the concatenated input with a block-diagonal weight:
+    nothing mixes between groups, dX stays per group."""
+    G, m, k, n, r = 2, 4, 3, 5, 2
+    x = rng_int(5, (G, m, k)); U = rng_int(6, (G, k, r)); V = rng_int(7, (G, n, r)); dY = rng_int(8, (G, m, n))
+    W = np.zeros((G * k, G * n))
+    for g in range(G):
+        W[g * k:(g + 1) * k, g * n:(g + 1) * n] = U[g] @ V[g].T
+    x_cat = np.concatenate(list(x), axis=1)
+    y, _ = oracle.linear_grouped_fwd(x, U, V)
+    np.testing.assert_array_equal(np.concatenate(list(y), axis=1), x_cat @ W)
+    dX, dU, dV = oracle.linear_grouped_bwd(x, U, V, dY)
+    np.testing.assert_array_equal(np.concatenate(list(dX), axis=1), np.concatenate(list(dY), axis=1) @ W.T)
+    for g in range(G):   # a group alone gives the same factor gradients
+        _, dU1, dV1 = oracle.linear_bwd(x[g], U[g], V[g], dY[g])
+        np.testing.assert_array_equal(dU[g], dU1)
+        np.testing.assert_array_equal(dV[g], dV1)
+
+
+def test_grouped_parameter_count_matches_the_lstm_table():
+    """Per-gate factorization of one LSTM layer: 8 factor pairs of 1500 x 375 / 375 x 1500 (Table 1:
+    4dr + 12hr parameters with d = h = 1500, r = 375)."""
+    d = h = 1500
+    r = 375
+    assert 8 * r * (d + h) == 4 * d * r + 12 * h * r
