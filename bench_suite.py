@@ -142,6 +142,65 @@ def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32, librar
             "tflops": 3 * flops_fwd / tot / 1e6, "gbs": (bytes_fwd + bytes_bwd) / tot / 1e3}
 
 
+def grouped_config(name, G, m, k, n, r, pk, shared_x, iters=24, repeats=5):
+    """G factorized layers of one shape in one call (row pitches padded to 16 bytes), beside the
+    same G layers issued one by one through the ungrouped calls."""
+    tdt = torch.bfloat16
+    up = lambda v: (v + 7) // 8 * 8
+    foot = 2 * G * (2 * m * up(k) + 2 * m * up(n) + m * up(r))
+    nsets = max(1, min(8, math.ceil(4 * L2_BYTES / foot)))
+    sig = 1.0 / math.sqrt(k)
+
+    def t3(g, rows, cols, scale=1.0):
+        buf = torch.zeros((g, rows, up(cols)), device="cuda", dtype=tdt)
+        buf[..., :cols] = (torch.randn((g, rows, cols), device="cuda") * scale).to(tdt)
+        return buf[..., :cols]
+
+    U, V = t3(G, k, r, sig), t3(G, n, r, sig)
+    stream = torch.cuda.current_stream()
+    sets, singles = [], []
+    for _ in range(nsets):
+        x = t3(1, m, k)[0] if shared_x else t3(G, m, k)
+        dY = t3(G, m, n)
+        y, T = t3(G, m, n), t3(G, m, r)
+        dX = t3(1, m, k)[0] if shared_x else t3(G, m, k)
+        dU, dV = t3(G, k, r), t3(G, n, r)
+        code = pf.PF_BF16
+        wf = torch.empty(max(256, pf.pf_lowrank_linear_grouped_workspace(G, m, k, n, r, code, 0)), dtype=torch.uint8, device="cuda")
+        wb = torch.empty(max(256, pf.pf_lowrank_linear_grouped_workspace(G, m, k, n, r, code, 1)), dtype=torch.uint8, device="cuda")
+        f, _ = pf.pf_lowrank_linear_grouped_fwd(x, U, V, y=y, T_stash=T, workspace=wf, stream=stream, prepare=True)
+        b, _ = pf.pf_lowrank_linear_grouped_bwd(x, U, V, dY, T_stash=T, dX=dX, dU=dU, dV=dV, workspace=wb, stream=stream,
+                                                prepare=True)
+        sets.append((f, b))
+        # the same layers one call per group (dX of a shared input would still have to be summed)
+        w1f = torch.empty(max(256, pf.pf_lowrank_linear_workspace(m, k, n, r, code, 0)), dtype=torch.uint8, device="cuda")
+        w1b = torch.empty(max(256, pf.pf_lowrank_linear_workspace(m, k, n, r, code, 1)), dtype=torch.uint8, device="cuda")
+        dXg = t3(G, m, k)
+        fs = [pf.pf_lowrank_linear_fwd(x if shared_x else x[g], U[g], V[g], y=y[g], T_stash=T[g], workspace=w1f,
+                                       stream=stream, prepare=True)[0] for g in range(G)]
+        bs = [pf.pf_lowrank_linear_bwd(x if shared_x else x[g], U[g], V[g], dY[g], T_stash=T[g], dX=dXg[g], dU=dU[g],
+                                       dV=dV[g], workspace=w1b, stream=stream, prepare=True)[0] for g in range(G)]
+        singles.append(((lambda fs=fs: [c() for c in fs]), (lambda bs=bs: [c() for c in bs])))
+    l0 = pf.pf_launch_count()
+    for c in sets[0]:
+        c()
+    launches = pf.pf_launch_count() - l0
+    t = _time(sets, iters, repeats=repeats)
+    t1 = _time(singles, max(2, iters // 4), repeats=repeats)
+    flops_fwd = 2.0 * G * m * r * (k + n)
+    xg = 1 if shared_x else G
+    bytes_fwd = 2 * (xg * m * k + G * m * n + G * r * (k + n))
+    bytes_bwd = 2 * (G * m * n + 2 * xg * m * k + 2 * G * r * (k + n))
+    ff, fb = _floors(flops_fwd, bytes_fwd, bytes_bwd, pk)
+    tot = t[-1]["median_us"]
+    return {"config": name, "kind": "grouped linear", "groups": G, "m": m, "k": k, "n": n, "r": r, "dtype": "bf16",
+            "shared_x": shared_x, "pitch": "padded to 16 B", "buffer_sets": nsets, "launches_fwd_bwd": launches,
+            "fwd_us": t[0]["median_us"], "bwd_us": t[1]["median_us"], "fwd_bwd_us": tot,
+            "one_call_per_group_fwd_bwd_us": t1[-1]["median_us"],
+            "floor_fwd_us": ff, "floor_bwd_us": fb, "roofline_frac": (ff + fb) / tot,
+            "tflops": 3 * flops_fwd / tot / 1e6, "gbs": (bytes_fwd + bytes_bwd) / tot / 1e3}
+
+
 def conv_config(name, c, pk, iters=20, repeats=5):
     tdt = torch.bfloat16
     M = c.N * c.H * c.W
@@ -214,11 +273,15 @@ def quick(pk):
             "fwd_us": round(r["fwd_us"], 2), "bwd_us": round(r["bwd_us"], 2), "fwd_bwd_us": round(r["fwd_bwd_us"], 2),
             "floor_us": round(r["floor_fwd_us"] + r["floor_bwd_us"], 2), "roofline_frac": round(r["roofline_frac"], 4),
             "launches": r.get("launches_fwd_bwd", r.get("launches_fwd_bwd_pack"))}
+        if "one_call_per_group_fwd_bwd_us" in r:
+            out[r["config"]]["one_call_per_group_fwd_bwd_us"] = round(r["one_call_per_group_fwd_bwd_us"], 2)
 
     keep(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk, iters=24, library=False, repeats=3))
     keep(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk, iters=24, library=False, repeats=3))
     keep(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, iters=24, library=False, repeats=3))
     keep(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True, iters=24, library=False, repeats=3))
+    keep(grouped_config("LSTM layer per gate (8 x 1500->1500 r375, m=700, shared x)", 8, 700, 1500, 1500, 375, pk, True, iters=12, repeats=3))
+    keep(grouped_config("attention projections (4 x 512->512 r128, m=8192)", 4, 8192, 512, 512, 128, pk, False, iters=12, repeats=3))
     for name, c in wl.conv_cases().items():
         keep(conv_config(f"{name} conv", c, pk, iters=8, repeats=3))
     for r in (128, 512):
@@ -256,6 +319,12 @@ def run(path, pk, only=None, iters=None, repeats=5, library=True):
         emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, iters=it(32), **lin))
     if want("C3 LSTM gates padded"):
         emit(linear_config("C3 LSTM gates", 700, 1500, 6000, 375, wl.BF16, pk, pad_pitch=True, iters=it(32), **lin))
+    if want("grouped LSTM per gate"):
+        emit(grouped_config("grouped LSTM per gate (8 x 1500->1500 r375, m=700, shared x)", 8, 700, 1500, 1500, 375, pk, True,
+                            iters=it(24), repeats=repeats))
+    if want("grouped attention projections"):
+        emit(grouped_config("grouped attention projections (4 x 512->512 r128, m=8192)", 4, 8192, 512, 512, 128, pk, False,
+                            iters=it(24), repeats=repeats))
     for name, c in wl.conv_cases().items():
         if want(f"{name} conv"):
             emit(conv_config(f"{name} conv", c, pk, iters=it(20), repeats=repeats))
