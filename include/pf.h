@@ -246,6 +246,17 @@ int pf_pack_factor_grads(const void* const* grads, const int64_t* numels, int co
                          void* flat, int64_t flat_capacity_elems, int64_t* offsets_out,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The inverse of pf_pack_factor_grads, for the step after the all-reduce of the flat buffer
+ * (Section 4.1: one buffer is communicated per iteration; every factor then needs its own averaged
+ * gradient back): tensor i receives flat[offsets_out[i] .. offsets_out[i] + numels[i]) bit for bit,
+ * with the same tight offsets (prefix sums of numels, written to offsets_out before return).
+ *   flat   device buffer of `flat_elems` elements (read only)
+ *   grads  host array of `count` device pointers (element-aligned), the destinations
+ * PF_ERR_WORKSPACE if the list is longer than flat_elems.  No workspace is needed. */
+int pf_unpack_factor_grads(const void* flat, int64_t flat_elems, void* const* grads, const int64_t* numels,
+                           int count, int dtype, int64_t* offsets_out,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

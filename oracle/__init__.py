@@ -14,6 +14,7 @@ Functions (paper passages they follow are cited in ``pf_oracle.c``):
     conv_fwd(x, U, V, stride, pad)   -> y, T            k x k conv to r channels, then 1 x 1
     conv_bwd(x, U, V, dY, stride, pad) -> dX, dU, dV
     pack(list_of_arrays)             -> flat, offsets   flat gradient buffer
+    unpack(flat, numels)             -> arrays, offsets its inverse
 
 Parity pins (tests/test_oracle_*.py): hand-computed tiny cases, the dense identity
 (xU)V^T = x(UV^T), special cases that reduce to a textbook matrix product or a library
@@ -176,6 +177,18 @@ def pack(grads):
     _load().pf_oracle_pack(ctypes.cast(ptrs, ctypes.c_void_p), _p(numels), count,
                            dt.itemsize, _p(flat), _p(offsets))
     return flat, offsets
+
+
+def unpack(flat, numels):
+    """The inverse of pack (Section 4.1, after the all-reduce): tensor i is the slice of the flat
+    buffer at the prefix-sum offset of numels.  Returns (list of arrays, offsets)."""
+    flat = np.asarray(flat)
+    offsets = np.zeros(len(numels) + 1, dtype=np.int64)
+    out = []
+    for i, cnt in enumerate(numels):
+        offsets[i + 1] = offsets[i] + int(cnt)
+        out.append(np.array([flat[e] for e in range(offsets[i], offsets[i + 1])], dtype=flat.dtype))
+    return out, offsets
 
 
 def rel_err(z, z_ref) -> float:

@@ -9,4 +9,4 @@ from .binding import (  # noqa: F401
     pf_lowrank_conv_fwd, pf_lowrank_conv_workspace, pf_lowrank_linear_bwd,
     pf_lowrank_linear_fwd, pf_lowrank_linear_fwd_static, pf_lowrank_linear_grouped_bwd,
     pf_lowrank_linear_grouped_fwd, pf_lowrank_linear_grouped_workspace, pf_lowrank_linear_workspace, pf_pack_factor_grads,
-    pf_static_scratch_bytes, pf_status_string, pf_version)
+    pf_static_scratch_bytes, pf_status_string, pf_unpack_factor_grads, pf_version)

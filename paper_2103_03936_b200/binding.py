@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.pf_lowrank_conv_bwd.argtypes = [vp] * 8 + [ci] * 11 + [vp, sz, vp]
         L.pf_pack_factor_grads.restype = ci
         L.pf_pack_factor_grads.argtypes = [vp, vp, ci, ci, vp, i64, vp, vp, sz, vp]
+        L.pf_unpack_factor_grads.restype = ci
+        L.pf_unpack_factor_grads.argtypes = [vp, i64, vp, vp, ci, ci, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -373,3 +375,22 @@ def pf_pack_factor_grads(grads, *, flat=None, stream=None, prepare=False):
                          (list(grads), flat)), (flat, offs)
     _check(lib().pf_pack_factor_grads(*args), "pf_pack_factor_grads")
     return flat, list(offs)
+
+
+def pf_unpack_factor_grads(flat, grads, *, stream=None):
+    """The inverse of pf_pack_factor_grads: tensor i of `grads` (contiguous CUDA tensors of flat's
+    dtype, overwritten) receives its slice of `flat`.  Returns the list of count+1 element offsets."""
+    count = len(grads)
+    offs = (ctypes.c_int64 * (count + 1))()
+    if count == 0:
+        _check(lib().pf_unpack_factor_grads(_ptr(flat), flat.numel(), None, None, 0, _dtype_code(flat), offs, None, 0,
+                                            _stream(stream)), "pf_unpack_factor_grads")
+        return [0]
+    for g in grads:
+        if not g.is_cuda or not g.is_contiguous() or g.dtype != flat.dtype:
+            raise ValueError("grads: contiguous CUDA tensors of flat's dtype")
+    numels = (ctypes.c_int64 * count)(*[g.numel() for g in grads])
+    ptrs = (ctypes.c_void_p * count)(*[g.data_ptr() for g in grads])
+    _check(lib().pf_unpack_factor_grads(_ptr(flat), flat.numel(), ptrs, numels, count, _dtype_code(flat), offs, None, 0,
+                                        _stream(stream)), "pf_unpack_factor_grads")
+    return list(offs)

@@ -573,4 +573,26 @@ int pf_pack_factor_grads(const void* const* grads, const int64_t* numels, int co
     return PF_OK;
 }
 
+int pf_unpack_factor_grads(const void* flat, int64_t flat_elems, void* const* grads, const int64_t* numels, int count,
+                           int dtype, int64_t* offsets_out, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream) {
+    (void)workspace; (void)workspace_bytes;
+    if (!valid_dtype(dtype) || count < 0 || !offsets_out || flat_elems < 0) return PF_ERR_INVALID_ARG;
+    if (count > 0 && (!grads || !numels)) return PF_ERR_INVALID_ARG;
+    offsets_out[0] = 0;
+    for (int i = 0; i < count; ++i) {
+        if (numels[i] < 0) return PF_ERR_INVALID_ARG;
+        if (numels[i] > 0 && (!grads[i] || !elem_aligned(grads[i], dtype))) return PF_ERR_INVALID_ARG;
+        if (numels[i] > (1LL << 46)) return PF_ERR_UNSUPPORTED;
+        offsets_out[i + 1] = offsets_out[i] + numels[i];
+    }
+    const int64_t total = offsets_out[count];
+    if (total > flat_elems) return PF_ERR_WORKSPACE;
+    if (total == 0) return PF_OK;
+    if (!flat || !elem_aligned(flat, dtype)) return PF_ERR_INVALID_ARG;
+    PF_CUDA(unpack_launch(flat, grads, numels, offsets_out, count, static_cast<int>(dtype_size(dtype)),
+                          static_cast<cudaStream_t>(cuda_stream)));
+    return PF_OK;
+}
+
 }  // extern "C"

@@ -104,6 +104,8 @@ cudaError_t repack_rows_bf16_multi(const RepackJob* jobs, int count, cudaStream_
 // pack
 cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const int64_t* offsets,
                         int count, int elem_bytes, void* flat, cudaStream_t stream);
+cudaError_t unpack_launch(const void* flat, void* const* grads, const int64_t* numels, const int64_t* offsets,
+                          int count, int elem_bytes, cudaStream_t stream);
 
 // The factorized linear forward behind pf_lowrank_linear_fwd and pf_lowrank_linear_fwd_static.
 // exact_need = false: the workspace must satisfy the public query; true: only the bytes the path

@@ -23,7 +23,7 @@ constexpr int kPackThreads = 256;
 
 struct PackBatch {
     const unsigned char* src[kPackBatch];
-    int64_t dst_byte[kPackBatch];   // destination byte offset in flat
+    unsigned char* dst[kPackBatch];  // where each tensor's bytes go
     int64_t bytes[kPackBatch];
     int chunk_prefix[kPackBatch + 1];
     int count;
@@ -43,7 +43,7 @@ __device__ __forceinline__ uint4 combine(const uint4 lo, const uint4 hi, unsigne
 }
 
 __global__ void __launch_bounds__(kPackThreads)
-pack_kernel(const PackBatch pb, unsigned char* __restrict__ flat) {
+pack_kernel(const PackBatch pb) {
     // which tensor does this chunk belong to?
     const int chunk = blockIdx.x;
     int lo = 0, hi = pb.count;  // invariant: prefix[lo] <= chunk < prefix[hi]
@@ -60,7 +60,7 @@ pack_kernel(const PackBatch pb, unsigned char* __restrict__ flat) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const unsigned char* src = pb.src[t];
     const int64_t bytes = pb.bytes[t];
-    unsigned char* dst = flat + pb.dst_byte[t];
+    unsigned char* dst = pb.dst[t];
     const int es = pb.elem_bytes;
 
     // destination split
@@ -114,8 +114,10 @@ pack_kernel(const PackBatch pb, unsigned char* __restrict__ flat) {
 
 }  // namespace
 
-cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const int64_t* offsets,
-                        int count, int elem_bytes, void* flat, cudaStream_t stream) {
+// One launch per kPackBatch tensors: tensor i moves numels[i] elements from src(i) to dst(i).
+template <typename SrcOf, typename DstOf>
+static cudaError_t copy_list(const int64_t* numels, int count, int elem_bytes, SrcOf src_of, DstOf dst_of,
+                             cudaStream_t stream) {
     int i = 0;
     while (i < count) {
         PackBatch pb;
@@ -127,8 +129,8 @@ cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const i
                 const int64_t bytes = numels[i] * elem_bytes;
                 const int64_t chunks = ceil_div(ceil_div(bytes, 16), kVecPerChunk);
                 if (pb.chunk_prefix[pb.count] + chunks > 0x7fffffff) return cudaErrorInvalidValue;
-                pb.src[pb.count] = static_cast<const unsigned char*>(grads[i]);
-                pb.dst_byte[pb.count] = offsets[i] * elem_bytes;
+                pb.src[pb.count] = src_of(i);
+                pb.dst[pb.count] = dst_of(i);
                 pb.bytes[pb.count] = bytes;
                 pb.chunk_prefix[pb.count + 1] = pb.chunk_prefix[pb.count] + static_cast<int>(chunks);
                 ++pb.count;
@@ -145,11 +147,29 @@ cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const i
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, pack_kernel, pb, static_cast<unsigned char*>(flat));
+        cudaError_t e = cudaLaunchKernelEx(&cfg, pack_kernel, pb);
         if (e != cudaSuccess) return e;
         count_launch();
     }
     return cudaSuccess;
+}
+
+cudaError_t pack_launch(const void* const* grads, const int64_t* numels, const int64_t* offsets,
+                        int count, int elem_bytes, void* flat, cudaStream_t stream) {
+    unsigned char* f = static_cast<unsigned char*>(flat);
+    return copy_list(numels, count, elem_bytes,
+                     [&](int i) { return static_cast<const unsigned char*>(grads[i]); },
+                     [&](int i) { return f + offsets[i] * elem_bytes; }, stream);
+}
+
+// The inverse: tensor i receives flat[offsets[i] .. offsets[i] + numels[i]).  The same kernel with
+// the roles swapped (the flat buffer is now the side that is only element-aligned).
+cudaError_t unpack_launch(const void* flat, void* const* grads, const int64_t* numels, const int64_t* offsets,
+                          int count, int elem_bytes, cudaStream_t stream) {
+    const unsigned char* f = static_cast<const unsigned char*>(flat);
+    return copy_list(numels, count, elem_bytes,
+                     [&](int i) { return f + offsets[i] * elem_bytes; },
+                     [&](int i) { return static_cast<unsigned char*>(grads[i]); }, stream);
 }
 
 }  // namespace pf

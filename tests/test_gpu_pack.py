@@ -74,3 +74,55 @@ def test_capacity_error_and_empty_list():
     assert e.value.status == 3
     flat, offs = pf.pf_pack_factor_grads([])
     assert offs == [0]
+
+
+def check_unpack(numels, dtype, seed=0, dst_shift=None, flat_shift=0):
+    """The inverse copy: bit-exact slices, guard bands around every destination; dst_shift / flat_shift
+    misalign the destinations and the flat buffer by elements."""
+    tensors_h = wl.pack_list(seed, numels, dtype)
+    flat_h, _ = oracle.pack(tensors_h)
+    total = int(sum(numels))
+    tdt = wl.to_torch(np.zeros(1, dtype=flat_h.dtype if total else np.uint16), dtype).dtype
+    pool = torch.zeros(total + flat_shift + 8, dtype=tdt, device="cuda")
+    if total:
+        pool[flat_shift:flat_shift + total] = dev(flat_h, dtype)
+    flat = pool[flat_shift:flat_shift + total]
+    guard = 16
+    bufs, dsts = [], []
+    for i, n in enumerate(numels):
+        sh = 0 if dst_shift is None else dst_shift[i % len(dst_shift)]
+        b = torch.full((n + sh + 2 * guard,), -7.0, dtype=tdt, device="cuda")
+        bufs.append((b, sh))
+        dsts.append(b[guard + sh:guard + sh + n])
+    offs = pf.pf_unpack_factor_grads(flat, dsts)
+    torch.cuda.synchronize()
+    want, want_offs = oracle.unpack(flat_h, numels)
+    assert offs == [int(o) for o in want_offs]
+    for (b, sh), d, w, n in zip(bufs, dsts, want, numels):
+        assert host(d, dtype).tobytes() == w.tobytes()
+        assert torch.all(b[:guard + sh] == -7.0) and torch.all(b[guard + sh + n:] == -7.0)
+
+
+@pytest.mark.parametrize("dtype", [wl.BF16, wl.F32])
+def test_unpack_small_lists_all_alignments(dtype):
+    check_unpack([1], dtype)
+    check_unpack([3, 5], dtype)
+    check_unpack([7, 0, 2, 1], dtype)
+    check_unpack([16, 1, 15, 33, 2, 64, 129, 5], dtype)
+    for shift in range(8):
+        check_unpack([37, 8, 101, 1, 64, 3], dtype, seed=shift, dst_shift=[shift, (3 * shift) % 8, 1], flat_shift=(5 * shift) % 8)
+
+
+def test_unpack_round_trip_at_model_scale():
+    numels = [147457, 16384, 589821, 65536, 1179653, 131072]
+    tensors = [torch.randn(n, device="cuda").to(torch.bfloat16) for n in numels]
+    flat, offs = pf.pf_pack_factor_grads(tensors)
+    back = [torch.full_like(t, -7.0) for t in tensors]
+    offs2 = pf.pf_unpack_factor_grads(flat, back)
+    torch.cuda.synchronize()
+    assert offs == offs2
+    for a, b in zip(tensors, back):
+        assert torch.equal(a, b)
+    with pytest.raises(pf.PfError) as e:          # a list longer than the flat buffer is refused
+        pf.pf_unpack_factor_grads(flat[:100], back)
+    assert e.value.status == 3

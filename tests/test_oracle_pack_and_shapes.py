@@ -109,3 +109,19 @@ def test_generator_distributions():
     small = wl.ConvCase("s", 2, 8, 8, c.C, c.R, c.O, wl.F32, c.seed).generate()
     assert small["x"].min() == 0.0 and (small["x"] == 0).mean() > 0.4      # post-ReLU
     assert abs(small["U"].std() - (2.0 / (9 * c.C)) ** 0.5) < 2e-3          # Kaiming fan-in
+
+
+@pytest.mark.parametrize("numels", [[1], [3, 5], [7, 0, 2, 1], [16, 1, 15, 33, 2]])
+@pytest.mark.parametrize("dt", [np.uint16, np.float32])
+def test_unpack_is_the_inverse_of_pack(numels, dt):
+    rng = np.random.default_rng(2)
+    grads = [rng.integers(0, 60000, size=n).astype(dt) for n in numels]
+    flat, offs = oracle.pack(grads)
+    back, offs2 = oracle.unpack(flat, numels)
+    np.testing.assert_array_equal(offs, offs2)
+    assert len(back) == len(grads)
+    for b, g in zip(back, grads):
+        assert b.dtype == dt and b.tobytes() == g.tobytes()
+    # and slicing by the prefix sums (the definition) gives the same
+    for i, b in enumerate(back):
+        np.testing.assert_array_equal(b, flat[offs[i]:offs[i + 1]])
