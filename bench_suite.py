@@ -269,12 +269,13 @@ def quick(pk):
     out = {}
 
     def keep(r):
-        out[r["config"] + (" (16 B pitches)" if r.get("pitch") == "padded to 16 B" else "")] = {
+        key = r["config"] + (" (16 B pitches)" if r.get("pitch") == "padded to 16 B" else "")
+        out[key] = {
             "fwd_us": round(r["fwd_us"], 2), "bwd_us": round(r["bwd_us"], 2), "fwd_bwd_us": round(r["fwd_bwd_us"], 2),
             "floor_us": round(r["floor_fwd_us"] + r["floor_bwd_us"], 2), "roofline_frac": round(r["roofline_frac"], 4),
             "launches": r.get("launches_fwd_bwd", r.get("launches_fwd_bwd_pack"))}
         if "one_call_per_group_fwd_bwd_us" in r:
-            out[r["config"]]["one_call_per_group_fwd_bwd_us"] = round(r["one_call_per_group_fwd_bwd_us"], 2)
+            out[key]["one_call_per_group_fwd_bwd_us"] = round(r["one_call_per_group_fwd_bwd_us"], 2)
 
     keep(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk, iters=24, library=False, repeats=3))
     keep(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk, iters=24, library=False, repeats=3))

@@ -149,22 +149,6 @@ __device__ __forceinline__ void gemm_tile(const CUtensorMap& tmA, const CUtensor
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    // While the previous kernel of the stream finishes, ask L2 for this block's first tiles (a prefetch
-    // only moves lines into L2, the point of coherence: harmless even if that kernel still writes them).
-    if (p.conv_mode == 0 && !grouped && (warp == 0 || warp == 6) && elect_one()) {
-        for (int i = 0; i < 6 && i < nkb; ++i) {
-            const int k0 = (kb_beg + i) * kBK;
-            if (warp == 0) {
-                if (p.a_mn) { tma_prefetch_l2_2d(&tmA, m0, k0); tma_prefetch_l2_2d(&tmA, m0 + 64, k0); }
-                else tma_prefetch_l2_2d(&tmA, k0, m0);
-            } else if (p.b_mn) {
-#pragma unroll
-                for (int h = 0; h < BN / 64; ++h) tma_prefetch_l2_2d(&tmB, n0 + 64 * h, k0);
-            } else {
-                tma_prefetch_l2_2d(&tmB, k0, n0);
-            }
-        }
-    }
     // A product marked independent reads nothing that the kernel launched just before it writes, so
     // it does not wait for that kernel: its blocks run beside it on SMs that kernel leaves free.  (Every
     // kernel of this library lets its successor start only after its own wait has returned, i.e. once
@@ -713,27 +697,24 @@ void pick_pair_splits(int64_t Mu, int64_t Mv, int64_t N, int64_t K, int kblock, 
 }
 
 // Slices of dU (k x r) and dV (n x r) in the backward of the linear layer, and whether dV runs BESIDE
-// the fused dX kernel instead of after it.  dV = dY^T T needs nothing that kernel writes, so when the
-// fused kernel leaves at least one SM per dV tile free, the dV blocks are sized to exactly those SMs,
-// come first in their launch and do not wait for the fused kernel; the dU blocks (which need G)
-// follow on the other SMs once that kernel's blocks retire.  When the contraction of the fused kernel's
-// first product is long against its output (n >= 2k) it is left unsplit for this (`unsplit`: one
-// block per 128-row tile, no block repeats another's first product), which frees more SMs.
-// `fused_blocks` = blocks of the fused kernel with the column split it would choose by itself, 0 = no
-// fused kernel.
-void bwd_split_plan(int64_t m, int64_t k, int64_t n, int64_t r, int64_t fused_blocks, int* su, int* sv, bool* beside,
-                    bool* unsplit) {
+// the fused dX kernel instead of after it.  dV = dY^T T needs nothing that kernel writes.  When the
+// contraction of the fused kernel's first product is long against its output (n >= 2k), that kernel is
+// left unsplit (one block per 128-row tile, no block repeats another's first product), which leaves
+// SMs free; the dV blocks are sized to exactly those SMs, come first in their launch and do not wait
+// for the fused kernel, and the dU blocks (which need G) follow on the other SMs once that kernel's
+// blocks retire.  (Measured on the Transformer-FFN shapes: doing the same for n < 2k, where only the
+// 20 SMs the split fused kernel leaves idle are free, loses more through the long dV blocks than the
+// overlap gains.)
+void bwd_split_plan(int64_t m, int64_t k, int64_t n, int64_t r, bool fused_dx, int* su, int* sv, bool* beside) {
     pick_pair_splits(k, n, r, m, kBK, su, sv);
     *beside = false;
-    *unsplit = false;
-    if (fused_blocks <= 0) return;
+    if (!fused_dx || n < 2 * k) return;
     const int bn = pick_bn(r);
     const int64_t row_tiles = ceil_div(m, kBM), nkb = ceil_div(m, kBK);
     const int64_t tu = ceil_div(k, kBM) * ceil_div(r, bn), tv = ceil_div(n, kBM) * ceil_div(r, bn);
-    const bool force = n >= 2 * k;
-    const int64_t free_sms = num_sms() - (force ? row_tiles : fused_blocks);
+    const int64_t free_sms = num_sms() - row_tiles;
     const int64_t smax = std::max<int64_t>(1, std::min<int64_t>(64, nkb / 4));
-    if (free_sms < tv || tu > num_sms() || tu > kFixTiles || tv > kFixTiles) return;
+    if (free_sms < tv || tu > kFixTiles || tv > kFixTiles) return;
     const int64_t b = std::min(free_sms / tv, smax);
     // dU gets the SMs that dV does not hold: dV may still be running when the fused kernel retires
     const int64_t a = std::min((num_sms() - tv * b) / tu, smax);
@@ -741,7 +722,6 @@ void bwd_split_plan(int64_t m, int64_t k, int64_t n, int64_t r, int64_t fused_bl
     *su = static_cast<int>(a);
     *sv = static_cast<int>(b);
     *beside = true;
-    *unsplit = force;
 }
 
 // C[M,N] (bf16, ldc) = A * B.  `partial` must hold splits*M*N floats when splits > 1.
@@ -981,20 +961,12 @@ size_t repack_room(int64_t rows, int64_t cols) {
 // Room for the fp32 slices of dU and dV under either backward structure (which one a call takes
 // depends on pointers the workspace query does not see): no block count exceeds one per SM per product.
 void bwd_partial_bytes(int64_t m, int64_t k, int64_t n, int64_t r, size_t* bytes_u, size_t* bytes_v) {
-    int su, sv;
-    bool beside, unsplit;
-    bwd_split_plan(m, k, n, r, 0, &su, &sv, &beside, &unsplit);
-    size_t bu = partial_bytes(k, r, su), bv = partial_bytes(n, r, sv);
-    ChainPlan plan;
-    if (use_chain(m, r) && chain_plan(m, n, k, r, true, &plan)) {
-        for (int64_t fused_blocks : {static_cast<int64_t>(plan.row_tiles) * plan.nsplit, static_cast<int64_t>(plan.row_tiles)}) {
-            bwd_split_plan(m, k, n, r, fused_blocks, &su, &sv, &beside, &unsplit);
-            bu = std::max(bu, partial_bytes(k, r, su));
-            bv = std::max(bv, partial_bytes(n, r, sv));
-        }
-    }
-    *bytes_u = align_up(bu, 256);
-    *bytes_v = align_up(bv, 256);
+    int su, sv, su2, sv2;
+    bool beside;
+    bwd_split_plan(m, k, n, r, false, &su, &sv, &beside);
+    bwd_split_plan(m, k, n, r, true, &su2, &sv2, &beside);
+    *bytes_u = align_up(std::max(partial_bytes(k, r, su), partial_bytes(k, r, su2)), 256);
+    *bytes_v = align_up(std::max(partial_bytes(n, r, sv), partial_bytes(n, r, sv2)), 256);
 }
 
 }  // namespace
@@ -1124,9 +1096,8 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     const bool fused_dx = use_chain(a.m, a.r) && (!a.dX || tma_ok(a.dX, a.lddx)) &&
                           chain_plan(a.m, a.n, a.k, a.r, a.dX != nullptr, &plan);
     int su, sv;
-    bool dv_beside, chain_unsplit;
-    bwd_split_plan(a.m, a.k, a.n, a.r, fused_dx ? static_cast<int64_t>(plan.row_tiles) * plan.nsplit : 0, &su, &sv, &dv_beside,
-                   &chain_unsplit);
+    bool dv_beside;
+    bwd_split_plan(a.m, a.k, a.n, a.r, fused_dx, &su, &sv, &dv_beside);
     bwd_partial_bytes(a.m, a.k, a.n, a.r, &pu_bytes, &pv_bytes);
     float* pu = reinterpret_cast<float*>(scratch);
     scratch += pu_bytes;
@@ -1142,7 +1113,7 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     bool dx_pending = false;     // dX still to be computed as a plain product G U^T
     if (fused_dx) {
         st = chain(dY.p, dY.ld, a.m, a.n, V.p, V.ld, a.r, U.p, U.ld, a.k, a.dX, a.lddx, G, ldG, a.stream, nullptr,
-                   chain_unsplit ? 1 : 0);
+                   dv_beside ? 1 : 0);
         if (st != PF_OK) return st;
     } else {
         // Few rows: G = dY V is a contraction split across blocks, and dV = dY^T T, which needs nothing
