@@ -41,7 +41,7 @@ class Guarded:
             assert torch.all(pad == -7.0), "row padding overwritten"
 
 
-# Every (case, tensor) that was judged by the cancellation rule below, in the order met.
+# Every (case, tensor) that took the cancellation rule below, in the order met.
 ESCAPES = []
 CANCELLED = 0.05      # a result counts as cancelled when ||exact|| < CANCELLED * ||summand magnitudes||
 

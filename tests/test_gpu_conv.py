@@ -59,7 +59,7 @@ SMALL = [  # N,H,W,C,R,O,k,stride,pad
 ]
 
 
-# bf16 outputs of the small shapes that may be judged against the magnitude of their summands
+# bf16 outputs of the small shapes that may be measured against the magnitude of their summands
 # (single near-cancelled sums, see _gpu.assert_close); fixed by the seeded inputs.
 MAX_CANCELLED_OUTPUTS = 1
 

@@ -63,7 +63,7 @@ def run_case(case, ld_pad=0, stash=True, need_dX=True, tiny=False, blocks=False)
 GRID = [(m, k, n, r) for m, k, n, r in itertools.product((1, 7, 130), (1, 17, 100), (3, 24, 130), (1, 5, 33))]
 
 
-# Outputs of the bf16 grid that may be judged against the magnitude of their summands (see
+# Outputs of the bf16 grid that may be measured against the magnitude of their summands (see
 # _gpu.assert_close): single near-cancelled sums.  The count is fixed by the seeded inputs.
 MAX_CANCELLED_OUTPUTS = 2
 
