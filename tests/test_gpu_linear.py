@@ -97,6 +97,15 @@ def test_fused_chain_envelope(m, k, n, r):
     run_case(wl.LinearCase("chain", m, k, n, r, wl.BF16, 14), stash=False, need_dX=False)
 
 
+@pytest.mark.parametrize("m,k,n,r", [(19500, 200, 128, 64), (40000, 136, 72, 100)])
+def test_fused_chain_more_row_tiles_than_sms(m, k, n, r):
+    """More 128-row tiles than SMs: the fused kernel runs as a persistent grid in which a CTA owns
+    several tiles (unequal counts, a ragged last tile) and the phases of consecutive tiles overlap;
+    forward (one and two output column tiles per row tile) and dX, with and without the stash."""
+    run_case(wl.LinearCase("multi", m, k, n, r, wl.BF16, 19))
+    run_case(wl.LinearCase("multi", m, k, n, r, wl.BF16, 20), stash=False, need_dX=False)
+
+
 @pytest.mark.parametrize("m,k,n,r", [(16000, 72, 264, 520), (9000, 200, 520, 392)])
 def test_wide_unfused_products_on_cta_pairs(m, k, n, r):
     """Ranks above 384 run as plain products; wide ones with many tiles use the two-CTA MMA kernel:
