@@ -142,6 +142,36 @@ def linear_config(name, m, k, n, r, dtype, pk, pad_pitch=False, iters=32, librar
             "tflops": 3 * flops_fwd / tot / 1e6, "gbs": (bytes_fwd + bytes_bwd) / tot / 1e3}
 
 
+def act_config(name, m, k, n, r, pk, iters=32, repeats=5):
+    """Forward with bias and max(0, .): the fused epilogue beside the plain forward and beside the plain
+    forward followed by the bias add and the activation as elementwise passes over y (torch, in place)."""
+    tdt = torch.bfloat16
+    foot = 2 * (m * k + m * n + m * r)
+    nsets = max(1, min(8, math.ceil(4 * L2_BYTES / foot)))
+    U, V = _rand((k, r), tdt, k ** -0.5), _rand((n, r), tdt, k ** -0.5)
+    b = _rand((n,), tdt, 0.5)
+    stream = torch.cuda.current_stream()
+    sets = []
+    for _ in range(nsets):
+        x = _rand((m, k), tdt)
+        y = torch.empty((m, n), dtype=tdt, device="cuda")
+        T = torch.empty((m, r), dtype=tdt, device="cuda")
+        f0, _ = pf.pf_lowrank_linear_fwd(x, U, V, y=y, T_stash=T, stream=stream, prepare=True)
+        f1, _ = pf.pf_lowrank_linear_fwd_act(x, U, V, bias=b, act=pf.PF_ACT_RELU, y=y, T_stash=T, stream=stream,
+                                             prepare=True)
+
+        def f2(f0=f0, y=y):
+            f0()
+            y.add_(b).relu_()
+        sets.append((f0, f1, f2))
+    t = _time(sets, iters, repeats=repeats)[:3]
+    bytes_fwd = 2 * (m * k + m * n + m * r + r * (k + n) + n)
+    return {"config": name, "kind": "act", "m": m, "k": k, "n": n, "r": r, "dtype": "bf16", "buffer_sets": nsets,
+            "plain_fwd_us": t[0]["median_us"], "fused_bias_relu_fwd_us": t[1]["median_us"],
+            "plain_fwd_plus_elementwise_us": t[2]["median_us"], "floor_fwd_us": bytes_fwd / pk["hbm_gbs"] / 1e3,
+            "roofline_frac": bytes_fwd / pk["hbm_gbs"] / 1e3 / t[1]["median_us"]}
+
+
 def grouped_config(name, G, m, k, n, r, pk, shared_x, iters=24, repeats=5):
     """G factorized layers of one shape in one call (row pitches padded to 16 bytes), beside the
     same G layers issued one by one through the ungrouped calls."""
@@ -314,6 +344,8 @@ def run(path, pk, only=None, iters=None, repeats=5, library=True):
         emit(linear_config("C1 tiny fp32", 64, 256, 256, 32, wl.F32, pk, iters=it(32), **lin))
     if want("C2a FFN up"):
         emit(linear_config("C2a FFN up", 8192, 512, 2048, 128, wl.BF16, pk, iters=it(32), **lin))
+    if want("C2a FFN up + bias + ReLU"):
+        emit(act_config("C2a FFN up + bias + ReLU (forward)", 8192, 512, 2048, 128, pk, iters=it(32), repeats=repeats))
     if want("C2b FFN down"):
         emit(linear_config("C2b FFN down", 8192, 2048, 512, 128, wl.BF16, pk, iters=it(32), **lin))
     if want("C3 LSTM gates tight"):

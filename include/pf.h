@@ -101,6 +101,30 @@ int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The forward with the bias and activation that follow the layer in a network:
+ *   y = act((x U) V^T + bias)
+ * the first half of the factorized feed-forward block FFN(x) = max(0, x W1 + b1) W2 + b2 with
+ * W1 = U1 V1^T (Section 2.4; biases are not factorized, Section 2.1), or, with PF_ACT_NONE, any
+ * factorized layer followed by its bias (the second half of the FFN, the LSTM gate pre-activations
+ * of Section 2.3).
+ *   bias [n] in `dtype`, contiguous; NULL = no bias.     act: PF_ACT_NONE or PF_ACT_RELU.
+ * bias and activation are applied to the fp32 result before the single rounding to `dtype` in the
+ * fused kernel (m >= 2048 rows at r <= 192, PF_BF16).  On the other paths y is first stored in
+ * `dtype` and a second pass adds the bias and applies the activation in place (two roundings for
+ * PF_BF16; one extra launch).  T_stash is x U as in pf_lowrank_linear_fwd (bias does not enter it).
+ * Same workspace, pitches and error behaviour as pf_lowrank_linear_fwd; an act outside the enum is
+ * PF_ERR_INVALID_ARG.  The backward of the activation (dY masked by y > 0) and the bias gradient
+ * (column sums of dY) are the caller's: pf_lowrank_linear_bwd takes the gradient of (x U) V^T. */
+typedef enum {
+    PF_ACT_NONE = 0,
+    PF_ACT_RELU = 1 /* max(0, .) */
+} pf_act;
+int pf_lowrank_linear_fwd_act(const void* x, int64_t ldx, const void* U, int64_t ldu,
+                              const void* V, int64_t ldv, const void* bias, int act,
+                              void* y, int64_t ldy, void* T_stash, int64_t ldt,
+                              int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* The same forward for callers that cannot allocate device memory and therefore have no
  * workspace to pass: latency-critical host paths where cudaMalloc is forbidden because it
  * synchronises the device, plug-ins that are handed tensors but no allocator, and processes

@@ -94,6 +94,20 @@ def linear_fwd(x, U, V):
     return y, T
 
 
+def linear_fwd_act(x, U, V, bias=None, relu=False):
+    """y = act((x U) V^T + bias), the factorized layer followed by its (unfactorized) bias and, for the
+    first half of the feed-forward block, max(0, .) (Section 2.4: FFN(x) = max(0, x W1 + b1) W2 + b2 with
+    W = U V^T; Section 2.1: biases stay as they are).  Returns (y, T) with T = x U."""
+    y, T = linear_fwd(x, U, V)
+    if bias is not None:
+        b = widen(bias)
+        assert b.shape == (y.shape[1],)
+        y = y + b[None, :]
+    if relu:
+        y = np.maximum(y, 0.0)
+    return y, T
+
+
 def linear_bwd(x, U, V, dY):
     x, U, V, dY = widen(x), widen(U), widen(V), widen(dY)
     m, k = x.shape

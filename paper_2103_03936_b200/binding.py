@@ -13,6 +13,7 @@ import os
 import torch
 
 PF_F32, PF_BF16 = 0, 1
+PF_ACT_NONE, PF_ACT_RELU = 0, 1
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libpf.so")
 _lib = None
@@ -44,6 +45,9 @@ def lib() -> ctypes.CDLL:
         L.pf_lowrank_linear_fwd.restype = ci
         L.pf_lowrank_linear_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                             i64, i64, i64, i64, ci, vp, sz, vp]
+        L.pf_lowrank_linear_fwd_act.restype = ci
+        L.pf_lowrank_linear_fwd_act.argtypes = [vp, i64, vp, i64, vp, i64, vp, ci, vp, i64, vp, i64,
+                                                i64, i64, i64, i64, ci, vp, sz, vp]
         L.pf_lowrank_linear_fwd_static.restype = ci
         L.pf_lowrank_linear_fwd_static.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                                    i64, i64, i64, i64, ci, vp]
@@ -168,6 +172,33 @@ def pf_lowrank_linear_fwd(x, U, V, *, y=None, T_stash=None, want_stash=False, wo
     if prepare:
         return _Prepared(lib().pf_lowrank_linear_fwd, args, "pf_lowrank_linear_fwd", (x, U, V, y, T_stash, ws)), out
     _check(lib().pf_lowrank_linear_fwd(*args), "pf_lowrank_linear_fwd")
+    return out
+
+
+def pf_lowrank_linear_fwd_act(x, U, V, *, bias=None, act=PF_ACT_NONE, y=None, T_stash=None, want_stash=False,
+                              workspace=None, stream=None, prepare=False):
+    """y = act((x U) V^T + bias); bias [n] in x's dtype or None, act PF_ACT_NONE / PF_ACT_RELU.
+    Otherwise as pf_lowrank_linear_fwd."""
+    dt = _dtype_code(x)
+    m, k = x.shape
+    n, r = V.shape
+    if U.shape != (k, r):
+        raise ValueError("U must be [k, r] and V [n, r]")
+    if bias is not None and (bias.shape != (n,) or bias.dtype != x.dtype or not bias.is_contiguous()):
+        raise ValueError("bias must be a contiguous [n] tensor of x's dtype")
+    if y is None:
+        y = torch.empty((m, n), dtype=x.dtype, device=x.device)
+    if T_stash is None and want_stash:
+        T_stash = torch.empty((m, r), dtype=x.dtype, device=x.device)
+    ws = _workspace(pf_lowrank_linear_workspace(m, k, n, r, dt, 0), x.device, workspace, stream)
+    args = (_ptr(x), _mat(x, "x"), _ptr(U), _mat(U, "U"), _ptr(V), _mat(V, "V"), _ptr(bias), int(act),
+            _ptr(y), _mat(y, "y"), _ptr(T_stash), _mat(T_stash, "T_stash") if T_stash is not None else 0,
+            m, k, n, r, dt, _ptr(ws), ws.numel(), _stream(stream))
+    out = (y, T_stash) if T_stash is not None else y
+    if prepare:
+        return _Prepared(lib().pf_lowrank_linear_fwd_act, args, "pf_lowrank_linear_fwd_act",
+                         (x, U, V, bias, y, T_stash, ws)), out
+    _check(lib().pf_lowrank_linear_fwd_act(*args), "pf_lowrank_linear_fwd_act")
     return out
 
 

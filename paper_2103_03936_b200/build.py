@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libpf.so")
-SOURCES = ["pf_api.cu", "pf_simt.cu", "pf_pack.cu", "pf_tc.cu", "pf_tc_chain.cu", "pf_tc_chain_multi.cu", "pf_tc_pair.cu", "pf_static.cu"]
+SOURCES = ["pf_api.cu", "pf_simt.cu", "pf_pack.cu", "pf_tc.cu", "pf_tc_chain.cu", "pf_tc_chain_multi.cu", "pf_tc_chain_act.cu", "pf_tc_pair.cu", "pf_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

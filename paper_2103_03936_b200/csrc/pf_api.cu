@@ -162,9 +162,11 @@ namespace pf {
 int linear_fwd_impl(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
                     int64_t ldv, void* y, int64_t ldy, void* T_stash, int64_t ldt,
                     int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
-                    void* workspace, size_t workspace_bytes, void* cuda_stream, bool exact_need) {
+                    void* workspace, size_t workspace_bytes, void* cuda_stream, bool exact_need, const void* bias,
+                    int act) {
     int st = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
     if (st != PF_OK) return st;
+    if ((act != PF_ACT_NONE && act != PF_ACT_RELU) || (bias && !elem_aligned(bias, dtype))) return PF_ERR_INVALID_ARG;
     if ((!y && m > 0) || ldy < n || !elem_aligned(y, dtype)) return PF_ERR_INVALID_ARG;
     if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
     const LinearWs w = linear_ws(m, k, n, r, dtype, false);
@@ -175,6 +177,7 @@ int linear_fwd_impl(const void* x, int64_t ldx, const void* U, int64_t ldu, cons
     a.y = y; a.ldy = ldy; a.T = T_stash; a.ldt = ldt;
     a.m = m; a.k = k; a.n = n; a.r = r;
     a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.stream = stream;
+    a.bias = bias; a.act = act;
     size_t need = w.total;
     if (exact_need) {
         bool tc_handles = false;
@@ -195,6 +198,7 @@ int linear_fwd_impl(const void* x, int64_t ldx, const void* U, int64_t ldu, cons
     const int64_t ldT = T_stash ? ldt : r;
     PF_CUDA(simt_gemm(mk(plainA(x, ldx, 1), plainB(U, ldu, 1), T, ldT, m, r, k, dtype), stream));
     PF_CUDA(simt_gemm(mk(plainA(T, ldT, 1), plainB(V, 1, ldv), y, ldy, m, n, r, dtype), stream));
+    PF_CUDA(bias_act_inplace(y, ldy, m, n, bias, act, dtype, stream));
     return PF_OK;
 }
 }  // namespace pf
@@ -207,6 +211,14 @@ int pf_lowrank_linear_fwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return linear_fwd_impl(x, ldx, U, ldu, V, ldv, y, ldy, T_stash, ldt, m, k, n, r, dtype, workspace, workspace_bytes,
                            cuda_stream, false);
+}
+
+int pf_lowrank_linear_fwd_act(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
+                              int64_t ldv, const void* bias, int act, void* y, int64_t ldy, void* T_stash, int64_t ldt,
+                              int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return linear_fwd_impl(x, ldx, U, ldu, V, ldv, y, ldy, T_stash, ldt, m, k, n, r, dtype, workspace, workspace_bytes,
+                           cuda_stream, false, bias, act);
 }
 
 int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,

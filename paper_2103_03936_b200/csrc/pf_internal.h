@@ -90,6 +90,9 @@ cudaError_t accumulate_f32(float* acc, const void* src, int64_t ld_src, int64_t 
                            cudaStream_t stream);
 cudaError_t round_out_f32(const float* acc, void* dst, int64_t ld_dst, int64_t rows, int64_t cols, int dtype,
                           cudaStream_t stream);
+// y = act(y + bias) in place: bias [cols] of the storage dtype or null, act 0 = identity, 1 = max(0, .)
+cudaError_t bias_act_inplace(void* y, int64_t ld, int64_t rows, int64_t cols, const void* bias, int act, int dtype,
+                             cudaStream_t stream);
 
 // Several such copies in one launch (row counts and widths below 2^31).
 struct RepackJob {
@@ -112,7 +115,8 @@ cudaError_t unpack_launch(const void* flat, void* const* grads, const int64_t* n
 // chosen for these pointers and pitches will touch.
 int linear_fwd_impl(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V, int64_t ldv, void* y,
                     int64_t ldy, void* T_stash, int64_t ldt, int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
-                    void* workspace, size_t workspace_bytes, void* cuda_stream, bool exact_need);
+                    void* workspace, size_t workspace_bytes, void* cuda_stream, bool exact_need,
+                    const void* bias = nullptr, int act = 0);
 
 // host-side count of kernels launched by this library
 void count_launch(int n = 1);

@@ -278,6 +278,32 @@ __global__ void round_out_kernel(const float* acc, T* dst, int64_t ld_dst, int64
         dst[rr * ld_dst + cc] = static_cast<T>(acc[i]);
     }
 }
+// y = act(y + bias) in place (the paths that do not fuse the epilogue into the producing kernel).
+template <typename T>
+__global__ void bias_act_kernel(T* y, int64_t ld, int64_t rows, int64_t cols, const T* bias, int act) {
+    const int64_t total = rows * cols;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t rr = i / cols, cc = i - rr * cols;
+        float v = static_cast<float>(y[rr * ld + cc]);
+        if (bias) v += static_cast<float>(bias[cc]);
+        if (act == 1) v = fmaxf(v, 0.f);
+        y[rr * ld + cc] = static_cast<T>(v);
+    }
+}
+cudaError_t bias_act_inplace(void* y, int64_t ld, int64_t rows, int64_t cols, const void* bias, int act, int dtype,
+                             cudaStream_t stream) {
+    const int64_t total = rows * cols;
+    if (total <= 0 || (!bias && !act)) return cudaSuccess;
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 8 * num_sms() ? ceil_div(total, 256) : 8 * num_sms());
+    if (dtype == PF_BF16)
+        bias_act_kernel<<<blocks, 256, 0, stream>>>(static_cast<__nv_bfloat16*>(y), ld, rows, cols,
+                                                    static_cast<const __nv_bfloat16*>(bias), act);
+    else
+        bias_act_kernel<<<blocks, 256, 0, stream>>>(static_cast<float*>(y), ld, rows, cols, static_cast<const float*>(bias), act);
+    count_launch();
+    return cudaGetLastError();
+}
 cudaError_t accumulate_f32(float* acc, const void* src, int64_t ld_src, int64_t rows, int64_t cols, int dtype, bool first,
                            cudaStream_t stream) {
     const int64_t total = rows * cols;

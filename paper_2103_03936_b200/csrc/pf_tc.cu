@@ -1041,7 +1041,7 @@ int linear_fwd(const LinearArgs& a, int* handled) {
     if (use_chain(a.m, a.r) && tma_ok(a.y, a.ldy) && chain_plan(a.m, a.k, a.n, a.r, true, &plan)) {
         // one fused kernel; the intermediate leaves the chip only if a stash was asked for
         st = chain(x.p, x.ld, a.m, a.k, U.p, U.ld, a.r, V.p, V.ld, a.n, a.y, a.ldy, a.T ? T : nullptr, ldT,
-                   a.stream);
+                   a.stream, nullptr, 0, a.bias, a.act);
     } else {
         float* p1 = reinterpret_cast<float*>(scratch + align_up(static_cast<size_t>(a.m) * pad8(a.r) * 2, 256));
         st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, T, ldT,
@@ -1049,6 +1049,10 @@ int linear_fwd(const LinearArgs& a, int* handled) {
                   (a.T && !stash_direct) ? a.T : nullptr, a.ldt, &stash_written);
         if (st != PF_OK) return st;
         st = gemm({T, ldT, false}, {V.p, V.ld, false}, a.m, a.n, a.r, a.y, a.ldy, 1, nullptr, a.stream);
+        // unfused products: bias and activation in a pass of their own over y
+        if (st == PF_OK && (a.bias || a.act) &&
+            bias_act_inplace(a.y, a.ldy, a.m, a.n, a.bias, a.act, PF_BF16, a.stream) != cudaSuccess)
+            return PF_ERR_CUDA;
     }
     if (st != PF_OK) return st;
     if (a.T && !stash_direct && !stash_written &&

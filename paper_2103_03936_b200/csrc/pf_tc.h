@@ -19,6 +19,8 @@ struct LinearArgs {
     int64_t m = 0, k = 0, n = 0, r = 0;
     char *ws = nullptr, *ws_T = nullptr, *ws_G = nullptr;
     cudaStream_t stream = nullptr;
+    const void* bias = nullptr;   // forward: y = act((x U) V^T + bias)
+    int act = 0;
 };
 
 struct ConvArgs {
@@ -45,7 +47,8 @@ struct ChainConv {
 };
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
-          cudaStream_t stream, const ChainConv* conv = nullptr, int max_split = 0);
+          cudaStream_t stream, const ChainConv* conv = nullptr, int max_split = 0, const void* bias = nullptr,
+          int act = 0);   // bias [N2] (bf16) and act (0 identity, 1 max(0, .)) apply to `out`
 
 // Plain product on CTA pairs (pf_tc_pair.cu); PF_ERR_UNSUPPORTED when the output is not 16-byte aligned
 // with a pitch that is a multiple of 8 elements.

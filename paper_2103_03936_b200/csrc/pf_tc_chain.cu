@@ -57,7 +57,7 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
 // out may be null (phase 1 only: T is written and nothing else).  All pointers must satisfy tma_ok.
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
-          cudaStream_t stream, const ChainConv* conv, int max_split) {
+          cudaStream_t stream, const ChainConv* conv, int max_split, const void* bias, int act) {
     ChainPlan plan;
     const int box_h = conv ? conv_box_h(conv->H, conv->W, 128) : 1;
     const int rows_tile = conv ? box_h * conv->W : 128;
@@ -98,8 +98,10 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
         grid_x = static_cast<int>(ceil_div(plan.row_tiles, per_cta));
         p.acc_base = 128; p.acc_bufs = 3;
     }
+    p.bias = bias; p.act = act;
     p.status = device_status_ptr();
     dim3 grid(static_cast<unsigned>(grid_x), static_cast<unsigned>(plan.nsplit), 1);
+    if (out && (bias || act)) return chain_launch_act(persistent, grid, plan.smem, stream, ta, tb1, tb2, to, tt, p);
     if (persistent) return chain_launch_multi(grid, plan.smem, stream, ta, tb1, tb2, to, tt, p);
     static bool configured[64] = {};
     int dev = 0;

@@ -52,6 +52,10 @@ struct ChainParams {
     int row_tiles;          // tiles along M; a CTA takes tiles blockIdx.x, blockIdx.x + gridDim.x, ...
     int acc_base, acc_bufs; // TMEM column of the first phase-2 accumulator and their number (4 on top of T's
                             // columns, or 3 behind them when tiles overlap)
+    // Output epilogue of the kEpi form: out = act(acc + bias), bias [N2] in bf16 (null = none),
+    // act 0 = identity, 1 = max(0, .); applied in fp32 before the single rounding to bf16.
+    const void* bias;
+    int act;
     unsigned int* status;
 };
 
@@ -84,6 +88,12 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* v) {
     return o;
 }
 
+__device__ __forceinline__ uint32_t relu_bf16x2(uint32_t w) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(w), "r"(0u));
+    return r;
+}
+
 // Position in the cycle of phase-2 accumulators: buffer index and its phase bit.
 struct AccPos {
     uint32_t b = 0, ph = 0;
@@ -102,7 +112,8 @@ struct RingPos {
 
 // kMulti: a CTA may own several row tiles (persistent grid); otherwise exactly the tile blockIdx.x, and
 // the loops over tiles below fold away at compile time.
-template <bool kMulti>
+// kEpi: the output epilogue adds a bias row and applies the activation (see ChainParams).
+template <bool kMulti, bool kEpi = false>
 __global__ void __launch_bounds__(kChainThreads, 1)
 tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB1,
                 const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmOut,
@@ -389,6 +400,28 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
             const int r0 = tile * p.rows_tile + q * 32;
             for (int j = 0; j < ntile; ++j) {
+                // kEpi: the bias of this warp's 64 columns, as 32 bf16 pairs per thread (every lane loads the
+                // same addresses: one broadcast transaction per load), fetched before the accumulator arrives
+                uint32_t bw[kEpi ? 32 : 1];
+                if constexpr (kEpi) {
+                    const int cb = (t_beg + j) * 128 + hcol * 64;
+                    const unsigned short* bp = reinterpret_cast<const unsigned short*>(p.bias);
+                    if (bp && cb + 64 <= p.N2 && (reinterpret_cast<uintptr_t>(bp) & 15) == 0) {
+                        const uint4* b4 = reinterpret_cast<const uint4*>(bp + cb);
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) {
+                            const uint4 w = __ldg(b4 + t);
+                            bw[4 * t] = w.x; bw[4 * t + 1] = w.y; bw[4 * t + 2] = w.z; bw[4 * t + 3] = w.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < 32; ++t) {
+                            const int c = cb + 2 * t;
+                            const uint32_t lo = (bp && c < p.N2) ? bp[c] : 0u, hi = (bp && c + 1 < p.N2) ? bp[c + 1] : 0u;
+                            bw[t] = lo | (hi << 16);
+                        }
+                    }
+                }
                 ok = mbar_wait_warp(smem_u32(&ctl->acc_full[ap.b]), ap.ph, abort_flag, p.status);
                 tc_fence_after();
                 if (!ok) break;
@@ -405,9 +438,22 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 __syncwarp();
                 ap.advance(NB);
+                if constexpr (kEpi) {
 #pragma unroll
-                for (int t = 0; t < 8; ++t)
-                    st_shared_v4(prow + ((static_cast<uint32_t>(t) ^ sw) << 4), pack8(v[t >> 2] + 8 * (t & 3)));
+                    for (int c = 0; c < 64; ++c) {
+                        const float b = __uint_as_float((c & 1) ? (bw[c >> 1] & 0xffff0000u) : (bw[c >> 1] << 16));
+                        v[c >> 5][c & 31] = __float_as_uint(__uint_as_float(v[c >> 5][c & 31]) + b);
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    uint4 o = pack8(v[t >> 2] + 8 * (t & 3));
+                    if constexpr (kEpi) {
+                        // max(0, .) commutes with the (monotonic) rounding, so it is taken on the rounded pairs
+                        if (p.act == 1) { o.x = relu_bf16x2(o.x); o.y = relu_bf16x2(o.y); o.z = relu_bf16x2(o.z); o.w = relu_bf16x2(o.w); }
+                    }
+                    st_shared_v4(prow + ((static_cast<uint32_t>(t) ^ sw) << 4), o);
+                }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
@@ -436,6 +482,10 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
 }  // namespace
 
+// Launch of the forms with the bias / activation epilogue (pf_tc_chain_act.cu).
+int chain_launch_act(bool persistent, dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& ta,
+                     const CUtensorMap& tb1, const CUtensorMap& tb2, const CUtensorMap& to, const CUtensorMap& tt,
+                     const ChainParams& p);
 // Launch of the persistent form (pf_tc_chain_multi.cu); same arguments as the kernel.
 int chain_launch_multi(dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& ta, const CUtensorMap& tb1,
                        const CUtensorMap& tb2, const CUtensorMap& to, const CUtensorMap& tt, const ChainParams& p);

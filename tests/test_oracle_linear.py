@@ -182,3 +182,58 @@ def test_grouped_parameter_count_matches_the_lstm_table():
     d = h = 1500
     r = 375
     assert 8 * r * (d + h) == 4 * d * r + 12 * h * r
+
+
+# ---- bias and activation after the factorized layer (Section 2.4: FFN(x) = max(0, x W1 + b1) W2 + b2)
+
+def test_bias_relu_hand_example():
+    """x = [1, -2], U = [[1], [1]] (T = -1), V = [[2], [-3]] gives (xU)V^T = [-2, 3]; with bias
+    [0.5, 0.5] that is [-1.5, 3.5], and max(0, .) leaves [0, 3.5]."""
+    x = np.array([[1.0, -2.0]], dtype=np.float32)
+    U = np.array([[1.0], [1.0]], dtype=np.float32)
+    V = np.array([[2.0], [-3.0]], dtype=np.float32)
+    b = np.array([0.5, 0.5], dtype=np.float32)
+    y, T = oracle.linear_fwd_act(x, U, V, b, relu=True)
+    np.testing.assert_array_equal(T, [[-1.0]])
+    np.testing.assert_array_equal(y, [[0.0, 3.5]])
+    y, _ = oracle.linear_fwd_act(x, U, V, b, relu=False)
+    np.testing.assert_array_equal(y, [[-1.5, 3.5]])
+    y, _ = oracle.linear_fwd_act(x, U, V, None, relu=True)
+    np.testing.assert_array_equal(y, [[0.0, 3.0]])
+
+
+@pytest.mark.parametrize("m,k,n,r", [(5, 7, 6, 3), (9, 4, 11, 4)])
+def test_bias_relu_equals_the_dense_ffn_half(m, k, n, r):
+    """max(0, x W + b) with the dense W = U V^T formed first (the other association order), in
+    integers so that both orders are exact; and the whole block FFN(x) = max(0, x W1 + b1) W2 + b2."""
+    x, U, V = rng_int(1, (m, k)), rng_int(2, (k, r)), rng_int(3, (n, r))
+    b = rng_int(4, (n,))
+    W = U.astype(np.float64) @ V.astype(np.float64).T
+    want = np.maximum(x.astype(np.float64) @ W + b, 0.0)
+    got, _ = oracle.linear_fwd_act(x, U, V, b, relu=True)
+    np.testing.assert_array_equal(got, want)
+    assert (got == 0).any() and (got > 0).any()          # the case exercises both branches
+    # second half of the block on top of it (no activation), against the dense formula
+    U2, V2, b2 = rng_int(5, (n, r)), rng_int(6, (k, r)), rng_int(7, (k,))
+    h = got.astype(np.float32)
+    ffn, _ = oracle.linear_fwd_act(h, U2, V2, b2, relu=False)
+    W2 = U2.astype(np.float64) @ V2.astype(np.float64).T
+    np.testing.assert_array_equal(ffn, want @ W2 + b2)
+
+
+def test_bias_relu_properties():
+    rng = np.random.default_rng(11)
+    x, U, V = (rng.standard_normal(s).astype(np.float32) for s in ((6, 5), (5, 3), (4, 3)))
+    b = rng.standard_normal(4).astype(np.float32)
+    y0, T0 = oracle.linear_fwd(x, U, V)
+    y1, T1 = oracle.linear_fwd_act(x, U, V, None, relu=False)
+    np.testing.assert_array_equal(y0, y1)                 # no bias, no activation: the plain layer
+    np.testing.assert_array_equal(T0, T1)
+    yb, _ = oracle.linear_fwd_act(x, U, V, b, relu=False)
+    np.testing.assert_allclose(yb - y0, np.broadcast_to(b.astype(np.float64), y0.shape), rtol=0, atol=1e-12)
+    yr, _ = oracle.linear_fwd_act(x, U, V, b, relu=True)
+    assert (yr >= 0).all()
+    np.testing.assert_array_equal(yr, np.where(yb > 0, yb, 0.0))
+    # positive homogeneity of max(0, .): scaling x and the bias by 4 (exact in binary) scales y by 4
+    y4, _ = oracle.linear_fwd_act(4 * x, U, V, 4 * b, relu=True)
+    np.testing.assert_array_equal(y4, 4 * yr)
