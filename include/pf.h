@@ -174,6 +174,31 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The same backward with two options for the factor gradients, as gradient accumulation over
+ * micro-batches and fp32 master gradients need them (the paper trains with mixed precision and
+ * all-reduces the factor gradients, Sections 4.1 and 3; it does not spell these variants out):
+ *   PF_GRAD_ACCUMULATE  dU and dV are ADDED to what the matrices hold: dU <- dU + x^T G, dV <- dV + dY^T (xU)
+ *                       (the caller zeroes them before the first micro-batch);
+ *   PF_GRAD_F32         dU [k, r] and dV [n, r] are fp32 matrices (lddu, lddv in floats) whatever
+ *                       `dtype` is: with PF_BF16 the fp32 sums are stored unrounded.
+ * dX is never accumulated and stays in `dtype`.  flags = 0 is pf_lowrank_linear_bwd.  The call runs
+ * the same kernels as the plain backward, with the plain gradients directed into the workspace, and
+ * one more small launch writes the caller's matrices: where a reduction over the batch was split across
+ * thread blocks (every benchmark shape) from the fp32 slices that reduction left in the workspace,
+ * summed again in the same order, so that the values are the unrounded fp32 sums (rounded once when
+ * added into a PF_BF16 matrix); on the remaining paths from the plain gradient (PF_BF16: the
+ * micro-batch's gradient has then been rounded to bf16 before it is widened or added).
+ * Same workspace query, pitches and errors as pf_lowrank_linear_bwd; unknown flag bits are
+ * PF_ERR_INVALID_ARG.  With m = 0 and PF_GRAD_ACCUMULATE nothing is written. */
+#define PF_GRAD_ACCUMULATE 1u
+#define PF_GRAD_F32 2u
+int pf_lowrank_linear_bwd_ex(const void* x, int64_t ldx, const void* U, int64_t ldu,
+                             const void* V, int64_t ldv, const void* dY, int64_t lddy,
+                             const void* T_stash, int64_t ldt,
+                             void* dX, int64_t lddx, void* dU, int64_t lddu, void* dV, int64_t lddv,
+                             int64_t m, int64_t k, int64_t n, int64_t r, int dtype, unsigned flags,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------
  * Grouped factorized fully-connected layers: `groups` layers of ONE shape (m, k, n, r), each with its
  * own factor pair (U_g, V_g), in one call -- the per-gate factorization of an LSTM layer

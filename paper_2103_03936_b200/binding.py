@@ -14,6 +14,7 @@ import torch
 
 PF_F32, PF_BF16 = 0, 1
 PF_ACT_NONE, PF_ACT_RELU = 0, 1
+PF_GRAD_ACCUMULATE, PF_GRAD_F32 = 1, 2
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libpf.so")
 _lib = None
@@ -56,6 +57,9 @@ def lib() -> ctypes.CDLL:
         L.pf_lowrank_linear_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                             vp, i64, vp, i64, vp, i64,
                                             i64, i64, i64, i64, ci, vp, sz, vp]
+        L.pf_lowrank_linear_bwd_ex.restype = ci
+        L.pf_lowrank_linear_bwd_ex.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
+                                               vp, i64, vp, i64, vp, i64, i64, i64, i64, i64, ci, ctypes.c_uint, vp, sz, vp]
         L.pf_lowrank_linear_grouped_workspace.restype = sz
         L.pf_lowrank_linear_grouped_workspace.argtypes = [ci, i64, i64, i64, i64, ci, ci]
         L.pf_lowrank_linear_grouped_fwd.restype = ci
@@ -225,22 +229,36 @@ def pf_lowrank_linear_fwd_static(x, U, V, *, y, T_stash=None, stream=None):
 
 
 def pf_lowrank_linear_bwd(x, U, V, dY, *, T_stash=None, need_dX=True, dX=None, dU=None, dV=None,
-                          workspace=None, stream=None, prepare=False):
-    """Returns (dX or None, dU, dV) for upstream gradient dY (prepare: see the forward)."""
+                          accumulate=False, grads_f32=False, workspace=None, stream=None, prepare=False):
+    """Returns (dX or None, dU, dV) for upstream gradient dY (prepare: see the forward).
+    accumulate: dU and dV (required then) are added to; grads_f32: dU and dV are fp32 tensors."""
     dt = _dtype_code(x)
     m, k = x.shape
     n, r = V.shape
+    flags = (PF_GRAD_ACCUMULATE if accumulate else 0) | (PF_GRAD_F32 if grads_f32 else 0)
+    gdt = torch.float32 if grads_f32 else x.dtype
+    if accumulate and (dU is None or dV is None):
+        raise ValueError("accumulate=True needs the dU and dV to add to")
     if dX is None and need_dX:
         dX = torch.empty((m, k), dtype=x.dtype, device=x.device)
     if dU is None:
-        dU = torch.empty((k, r), dtype=x.dtype, device=x.device)
+        dU = torch.empty((k, r), dtype=gdt, device=x.device)
     if dV is None:
-        dV = torch.empty((n, r), dtype=x.dtype, device=x.device)
+        dV = torch.empty((n, r), dtype=gdt, device=x.device)
+    if dU.dtype != gdt or dV.dtype != gdt:
+        raise ValueError("dU and dV must be float32 with grads_f32=True and of x's dtype otherwise")
     ws = _workspace(pf_lowrank_linear_workspace(m, k, n, r, dt, 1), x.device, workspace, stream)
     args = (_ptr(x), _mat(x, "x"), _ptr(U), _mat(U, "U"), _ptr(V), _mat(V, "V"), _ptr(dY), _mat(dY, "dY"),
             _ptr(T_stash), _mat(T_stash, "T_stash") if T_stash is not None else 0,
             _ptr(dX), _mat(dX, "dX") if dX is not None else 0, _ptr(dU), _mat(dU, "dU"),
             _ptr(dV), _mat(dV, "dV"), m, k, n, r, dt, _ptr(ws), ws.numel(), _stream(stream))
+    if flags:
+        args = args[:21] + (flags,) + args[21:]
+        if prepare:
+            return _Prepared(lib().pf_lowrank_linear_bwd_ex, args, "pf_lowrank_linear_bwd_ex",
+                             (x, U, V, dY, T_stash, dX, dU, dV, ws)), (dX, dU, dV)
+        _check(lib().pf_lowrank_linear_bwd_ex(*args), "pf_lowrank_linear_bwd_ex")
+        return dX, dU, dV
     if prepare:
         return _Prepared(lib().pf_lowrank_linear_bwd, args, "pf_lowrank_linear_bwd",
                          (x, U, V, dY, T_stash, dX, dU, dV, ws)), (dX, dU, dV)

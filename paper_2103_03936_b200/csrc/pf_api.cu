@@ -58,7 +58,7 @@ SimtGemm mk(const MatA& A, const MatB& B, void* C, int64_t ldc, int64_t M, int64
 
 // ------------------------------------------------------------------------------ linear
 struct LinearWs {
-    size_t off_T, off_G, off_partial, off_tc, total;
+    size_t off_T, off_G, off_partial, off_gtmp, off_tc, total;
     int splits_dU, splits_dV;
 };
 
@@ -75,6 +75,9 @@ LinearWs linear_ws(int64_t m, int64_t k, int64_t n, int64_t r, int dtype, bool b
         size_t pu = w.splits_dU > 1 ? static_cast<size_t>(w.splits_dU) * k * r * 4 : 0;
         size_t pv = w.splits_dV > 1 ? static_cast<size_t>(w.splits_dV) * n * r * 4 : 0;
         w.off_partial = off; off += align_up(pu > pv ? pu : pv, 256);
+        // plain dU and dV of a call that wants them in fp32 or accumulated, on the paths that cannot
+        // write them that way directly
+        w.off_gtmp = off; off += align_up(static_cast<size_t>(k) * r * s, 256) + align_up(static_cast<size_t>(n) * r * s, 256);
     }
     w.off_tc = off;
     if (dtype == PF_BF16) off += align_up(tc::linear_extra_workspace(m, k, n, r, bwd), 256);
@@ -226,11 +229,23 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
                           void* dX, int64_t lddx, void* dU, int64_t lddu, void* dV, int64_t lddv,
                           int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return pf_lowrank_linear_bwd_ex(x, ldx, U, ldu, V, ldv, dY, lddy, T_stash, ldt, dX, lddx, dU, lddu, dV, lddv, m, k, n, r,
+                                    dtype, 0u, workspace, workspace_bytes, cuda_stream);
+}
+
+int pf_lowrank_linear_bwd_ex(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
+                             int64_t ldv, const void* dY, int64_t lddy, const void* T_stash, int64_t ldt,
+                             void* dX, int64_t lddx, void* dU, int64_t lddu, void* dV, int64_t lddv,
+                             int64_t m, int64_t k, int64_t n, int64_t r, int dtype, unsigned flags,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
     int st = validate_linear_common(x, ldx, U, ldu, V, ldv, m, k, n, r, dtype);
     if (st != PF_OK) return st;
+    if (flags & ~static_cast<unsigned>(PF_GRAD_ACCUMULATE | PF_GRAD_F32)) return PF_ERR_INVALID_ARG;
+    const bool g_acc = (flags & PF_GRAD_ACCUMULATE) != 0, g_f32 = (flags & PF_GRAD_F32) != 0;
+    const int gdtype = g_f32 ? PF_F32 : dtype;          // storage type of dU and dV
     if ((!dY && m > 0) || lddy < n || !elem_aligned(dY, dtype)) return PF_ERR_INVALID_ARG;
-    if (!dU || lddu < r || !elem_aligned(dU, dtype)) return PF_ERR_INVALID_ARG;
-    if (!dV || lddv < r || !elem_aligned(dV, dtype)) return PF_ERR_INVALID_ARG;
+    if (!dU || lddu < r || !elem_aligned(dU, gdtype)) return PF_ERR_INVALID_ARG;
+    if (!dV || lddv < r || !elem_aligned(dV, gdtype)) return PF_ERR_INVALID_ARG;
     if (dX && (lddx < k || !elem_aligned(dX, dtype))) return PF_ERR_INVALID_ARG;
     if (T_stash && (ldt < r || !elem_aligned(T_stash, dtype))) return PF_ERR_INVALID_ARG;
     const LinearWs w = linear_ws(m, k, n, r, dtype, true);
@@ -238,12 +253,20 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
     if (st != PF_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t s = dtype_size(dtype);
-    if (m == 0) {  // empty sums
-        PF_CUDA(cudaMemset2DAsync(dU, lddu * s, 0, r * s, k, stream));
-        PF_CUDA(cudaMemset2DAsync(dV, lddv * s, 0, r * s, n, stream));
+    if (m == 0) {  // empty sums: zero, or nothing to add
+        if (g_acc) return PF_OK;
+        const size_t gs = dtype_size(gdtype);
+        PF_CUDA(cudaMemset2DAsync(dU, lddu * gs, 0, r * gs, k, stream));
+        PF_CUDA(cudaMemset2DAsync(dV, lddv * gs, 0, r * gs, n, stream));
         return PF_OK;
     }
     char* ws = static_cast<char*>(workspace);
+    // A call with gradient flags that no kernel can honour directly computes plain dU and dV into the
+    // workspace and adds / widens them into the caller's matrices in a pass of its own.
+    void* const user_dU = dU;
+    void* const user_dV = dV;
+    const int64_t user_lddu = lddu, user_lddv = lddv;
+    bool indirect = false;
 
     if (dtype == PF_BF16) {
         tc::LinearArgs a;
@@ -252,9 +275,40 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
         a.dX = dX; a.lddx = lddx; a.dU = dU; a.lddu = lddu; a.dV = dV; a.lddv = lddv;
         a.m = m; a.k = k; a.n = n; a.r = r;
         a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.ws_G = ws + w.off_G; a.stream = stream;
+        tc::LinearArgs::Slices su_info, sv_info;
+        if (flags) {
+            // plain gradients go to the workspace; where a reduction was split, its fp32 slices are still
+            // there afterwards and are summed once more, unrounded, into the caller's matrix
+            indirect = true;
+            dU = ws + w.off_gtmp; lddu = r;
+            dV = ws + w.off_gtmp + align_up(static_cast<size_t>(k) * r * s, 256); lddv = r;
+            a.dU = dU; a.lddu = lddu; a.dV = dV; a.lddv = lddv;
+            a.du_slices = &su_info; a.dv_slices = &sv_info;
+        }
         int handled = 0;
         st = tc::linear_bwd(a, &handled);
-        if (st != PF_OK || handled) return st;
+        if (st != PF_OK) return st;
+        if (handled && flags) {
+            SliceSums jobs[2];
+            int nj = 0;
+            if (su_info.splits > 1)
+                jobs[nj++] = SliceSums{su_info.partial, user_dU, user_lddu, static_cast<int>(k), static_cast<int>(r), su_info.splits,
+                                       su_info.bn, su_info.tiles_x, su_info.tiles_y, g_f32, g_acc};
+            else
+                PF_CUDA(grad_combine(user_dU, user_lddu, gdtype, dU, lddu, dtype, k, r, g_acc, stream));
+            if (sv_info.splits > 1)
+                jobs[nj++] = SliceSums{sv_info.partial, user_dV, user_lddv, static_cast<int>(n), static_cast<int>(r), sv_info.splits,
+                                       sv_info.bn, sv_info.tiles_x, sv_info.tiles_y, g_f32, g_acc};
+            else
+                PF_CUDA(grad_combine(user_dV, user_lddv, gdtype, dV, lddv, dtype, n, r, g_acc, stream));
+            if (nj) PF_CUDA(slices_to_gradients(jobs, nj, stream));
+            return PF_OK;
+        }
+        if (handled) return PF_OK;
+    } else if (flags) {
+        indirect = true;
+        dU = ws + w.off_gtmp; lddu = r;
+        dV = ws + w.off_gtmp + align_up(static_cast<size_t>(k) * r * s, 256); lddv = r;
     }
     const void* T = T_stash;
     int64_t ldT = ldt;
@@ -269,6 +323,10 @@ int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu
     if (dX) PF_CUDA(simt_gemm(mk(plainA(G, r, 1), plainB(U, 1, ldu), dX, lddx, m, k, r, dtype), stream));
     PF_CUDA(simt_gemm(mk(plainA(x, 1, ldx), plainB(G, r, 1), dU, lddu, k, r, m, dtype, w.splits_dU, partial), stream));
     PF_CUDA(simt_gemm(mk(plainA(dY, 1, lddy), plainB(T, ldT, 1), dV, lddv, n, r, m, dtype, w.splits_dV, partial), stream));
+    if (indirect) {
+        PF_CUDA(grad_combine(user_dU, user_lddu, gdtype, dU, lddu, dtype, k, r, g_acc, stream));
+        PF_CUDA(grad_combine(user_dV, user_lddv, gdtype, dV, lddv, dtype, n, r, g_acc, stream));
+    }
     return PF_OK;
 }
 

@@ -90,6 +90,19 @@ cudaError_t accumulate_f32(float* acc, const void* src, int64_t ld_src, int64_t 
                            cudaStream_t stream);
 cudaError_t round_out_f32(const float* acc, void* dst, int64_t ld_dst, int64_t rows, int64_t cols, int dtype,
                           cudaStream_t stream);
+// out (fp32 or the storage dtype, pitch ld_out) = (accumulate ? out : 0) + src (storage dtype src_dtype).
+cudaError_t grad_combine(void* out, int64_t ld_out, int out_dtype, const void* src, int64_t ld_src, int src_dtype,
+                         int64_t rows, int64_t cols, bool accumulate, cudaStream_t stream);
+// out = (accumulate ? out : 0) + the sum, in slice order, of the fp32 slices a split tensor-core reduction
+// left at `partial` ([tile][slice][128][bn], see pf_simt.cu); one launch for up to two matrices.
+struct SliceSums {
+    const float* partial;
+    void* out;          // fp32 (out_f32) or bf16 matrix, pitch ld in its own elements
+    long long ld;
+    int M, N, splits, bn, tiles_x, tiles_y;
+    bool out_f32, accumulate;
+};
+cudaError_t slices_to_gradients(const SliceSums* jobs, int count, cudaStream_t stream);
 // y = act(y + bias) in place: bias [cols] of the storage dtype or null, act 0 = identity, 1 = max(0, .)
 cudaError_t bias_act_inplace(void* y, int64_t ld, int64_t rows, int64_t cols, const void* bias, int act, int dtype,
                              cudaStream_t stream);

@@ -278,6 +278,97 @@ __global__ void round_out_kernel(const float* acc, T* dst, int64_t ld_dst, int64
         dst[rr * ld_dst + cc] = static_cast<T>(acc[i]);
     }
 }
+// out = (accumulate ? out : 0) + src, the sum taken in fp32 and rounded once to out's type.
+template <typename TO, typename TS>
+__global__ void grad_combine_kernel(TO* out, int64_t ld_out, const TS* src, int64_t ld_src, int64_t rows, int64_t cols,
+                                    int accumulate) {
+    const int64_t total = rows * cols;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t rr = i / cols, cc = i - rr * cols;
+        float v = static_cast<float>(src[rr * ld_src + cc]);
+        if (accumulate) v += static_cast<float>(out[rr * ld_out + cc]);
+        out[rr * ld_out + cc] = static_cast<TO>(v);
+    }
+}
+cudaError_t grad_combine(void* out, int64_t ld_out, int out_dtype, const void* src, int64_t ld_src, int src_dtype,
+                         int64_t rows, int64_t cols, bool accumulate, cudaStream_t stream) {
+    const int64_t total = rows * cols;
+    if (total <= 0) return cudaSuccess;
+    const int blocks = static_cast<int>(ceil_div(total, 256) < 8 * num_sms() ? ceil_div(total, 256) : 8 * num_sms());
+    const int acc = accumulate ? 1 : 0;
+    if (out_dtype == PF_F32 && src_dtype == PF_BF16)
+        grad_combine_kernel<<<blocks, 256, 0, stream>>>(static_cast<float*>(out), ld_out, static_cast<const __nv_bfloat16*>(src), ld_src, rows, cols, acc);
+    else if (out_dtype == PF_F32)
+        grad_combine_kernel<<<blocks, 256, 0, stream>>>(static_cast<float*>(out), ld_out, static_cast<const float*>(src), ld_src, rows, cols, acc);
+    else
+        grad_combine_kernel<<<blocks, 256, 0, stream>>>(static_cast<__nv_bfloat16*>(out), ld_out, static_cast<const __nv_bfloat16*>(src), ld_src, rows, cols, acc);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// The fp32 slices a split tensor-core reduction left in the workspace, summed once more in slice order
+// (the very sums the reduction rounded to bf16) and written unrounded to an fp32 matrix and / or added to
+// the old contents.  Slice layout: [tile][slice][128 rows][bn floats], tile = column tile * tiles_x + row
+// tile, the 16-byte pieces of a row XOR-permuted by the row index.
+struct SliceSumJob {
+    const float* partial;
+    void* out;
+    long long ld;
+    int M, N, S, bn, tiles_x, tiles_y, out_f32, accumulate;
+};
+__global__ void __launch_bounds__(256) slices_to_gradients_kernel(const SliceSumJob j0, const SliceSumJob j1, int blocks0) {
+    const bool first = static_cast<int>(blockIdx.x) < blocks0;
+    const SliceSumJob& j = first ? j0 : j1;
+    const int b = first ? blockIdx.x : blockIdx.x - blocks0;
+    const int nb = first ? blocks0 : gridDim.x - blocks0;
+    const int pieces = j.bn / 4;
+    const long long total = static_cast<long long>(j.tiles_x) * j.tiles_y * 128 * pieces;
+    for (long long i = static_cast<long long>(b) * blockDim.x + threadIdx.x; i < total; i += static_cast<long long>(nb) * blockDim.x) {
+        const int pc = static_cast<int>(i % pieces);
+        const long long t = i / pieces;
+        const int rin = static_cast<int>(t % 128);
+        const int tile = static_cast<int>(t / 128);
+        const int bx = tile % j.tiles_x, by = tile / j.tiles_x;
+        const int row = bx * 128 + rin, col = by * j.bn + pc * 4;
+        if (row >= j.M || col >= j.N) continue;
+        const float* src = j.partial + (static_cast<size_t>(tile) * j.S * 128 + rin) * j.bn + ((pc ^ (rin & (pieces - 1))) << 2);
+        float4 acc = *reinterpret_cast<const float4*>(src);
+        for (int s = 1; s < j.S; ++s) {
+            const float4 w = *reinterpret_cast<const float4*>(src + static_cast<size_t>(s) * 128 * j.bn);
+            acc.x += w.x; acc.y += w.y; acc.z += w.z; acc.w += w.w;
+        }
+        const float sums[4] = {acc.x, acc.y, acc.z, acc.w};
+        const size_t at = static_cast<size_t>(row) * j.ld + col;
+        for (int e = 0; e < 4 && col + e < j.N; ++e) {
+            if (j.out_f32) {
+                float* o = static_cast<float*>(j.out) + at + e;
+                *o = j.accumulate ? *o + sums[e] : sums[e];
+            } else {
+                __nv_bfloat16* o = static_cast<__nv_bfloat16*>(j.out) + at + e;
+                *o = __float2bfloat16_rn(j.accumulate ? __bfloat162float(*o) + sums[e] : sums[e]);
+            }
+        }
+    }
+}
+cudaError_t slices_to_gradients(const SliceSums* jobs, int count, cudaStream_t stream) {
+    if (count < 1 || count > 2) return cudaErrorInvalidValue;
+    SliceSumJob j[2];
+    int blocks[2] = {0, 0};
+    for (int i = 0; i < 2; ++i) {
+        const SliceSums& s = jobs[i < count ? i : 0];
+        j[i] = SliceSumJob{s.partial, s.out, s.ld, s.M, s.N, s.splits, s.bn, s.tiles_x, s.tiles_y, s.out_f32 ? 1 : 0, s.accumulate ? 1 : 0};
+        if (i < count) {
+            const long long total = static_cast<long long>(s.tiles_x) * s.tiles_y * 128 * (s.bn / 4);
+            blocks[i] = static_cast<int>(std::min<long long>(ceil_div(total, 256), 4LL * num_sms()));
+            if (blocks[i] < 1) blocks[i] = 1;
+        }
+    }
+    slices_to_gradients_kernel<<<blocks[0] + blocks[1], 256, 0, stream>>>(j[0], j[1], blocks[0]);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // y = act(y + bias) in place (the paths that do not fuse the epilogue into the producing kernel).
 template <typename T>
 __global__ void bias_act_kernel(T* y, int64_t ld, int64_t rows, int64_t cols, const T* bias, int act) {

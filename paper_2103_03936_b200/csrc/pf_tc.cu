@@ -1108,6 +1108,15 @@ int linear_bwd(const LinearArgs& a, int* handled) {
     float* pv = reinterpret_cast<float*>(scratch);
     scratch += pv_bytes;
     float* p1 = reinterpret_cast<float*>(scratch);
+    // the slices of the reductions as they will be launched (the last prepared product is the launched one)
+    auto note = [](LinearArgs::Slices* out, const GemmLaunch* g) {
+        if (!out) return;
+        *out = LinearArgs::Slices();
+        if (g && g->p.splits > 1) {
+            out->partial = g->p.partial; out->splits = g->p.splits; out->bn = g->bn;
+            out->tiles_x = static_cast<int>(g->grid.x); out->tiles_y = static_cast<int>(g->grid.y);
+        }
+    };
     // G = dY V ; dX = G U^T ; dU = x^T G ; dV = dY^T T
     if (need_T) {   // no stash: recompute T = x U
         st = gemm({x.p, x.ld, false}, {U.p, U.ld, true}, a.m, a.r, a.k, Tbuf, pad8(a.r),
@@ -1132,6 +1141,8 @@ int linear_bwd(const LinearArgs& a, int* handled) {
             ok = gemm_prepare({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, nullptr, &gx) == PF_OK;
         ok = ok && (gg.p.splits > 1 || gv.p.splits <= 1) && (gu.p.splits > 1 || !a.dX || gx.p.splits <= 1);
         if (ok) {
+            note(a.du_slices, &gu);
+            note(a.dv_slices, &gv);
             const GemmLaunch* first[2] = {&gg, &gv};
             st = gemm_multi(first, 2, a.stream);
             if (st == PF_OK) {
@@ -1156,6 +1167,8 @@ int linear_bwd(const LinearArgs& a, int* handled) {
         if (ok && dx_pending)
             ok = gemm_prepare({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, nullptr, &gx) == PF_OK;
         if (ok) {
+            note(a.du_slices, &gu);
+            note(a.dv_slices, &gv);
             const GemmLaunch* list[3] = {&gu, &gv, &gx};
             // a split product has to come before the plain ones
             if (gu.p.splits <= 1 && gv.p.splits > 1) { list[0] = &gv; list[1] = &gu; }
@@ -1183,6 +1196,8 @@ int linear_bwd(const LinearArgs& a, int* handled) {
         st = gemm({G, ldG, false}, {U.p, U.ld, false}, a.m, a.k, a.r, a.dX, a.lddx, 1, nullptr, a.stream);
         if (st != PF_OK) return st;
     }
+    note(a.du_slices, nullptr);      // launched by gemm(), which may choose other kernels and slice counts
+    note(a.dv_slices, nullptr);
     st = gemm({x.p, x.ld, true}, {G, ldG, true}, a.k, a.r, a.m, a.dU, a.lddu, su, pu, a.stream);
     if (st != PF_OK) return st;
     return gemm({dY.p, dY.ld, true}, {T.p, T.ld, true}, a.n, a.r, a.m, a.dV, a.lddv, sv, pv, a.stream);

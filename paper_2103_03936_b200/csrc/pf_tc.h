@@ -21,6 +21,15 @@ struct LinearArgs {
     cudaStream_t stream = nullptr;
     const void* bias = nullptr;   // forward: y = act((x U) V^T + bias)
     int act = 0;
+    // backward: where the fp32 slices of dU / dV were left in the workspace (filled in when the reduction
+    // over the batch was split across thread blocks; splits <= 1 otherwise), for callers that want the
+    // unrounded sums
+    struct Slices {
+        const float* partial = nullptr;
+        int splits = 0, bn = 0, tiles_x = 0, tiles_y = 0;
+    };
+    Slices* du_slices = nullptr;
+    Slices* dv_slices = nullptr;
 };
 
 struct ConvArgs {
