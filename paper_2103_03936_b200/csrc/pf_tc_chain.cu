@@ -102,6 +102,21 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
     p.status = device_status_ptr();
     dim3 grid(static_cast<unsigned>(grid_x), static_cast<unsigned>(plan.nsplit), 1);
     if (out && (bias || act)) return chain_launch_act(persistent, grid, plan.smem, stream, ta, tb1, tb2, to, tt, p);
+    if (persistent && plan.r_pad <= 128) {
+        // software-pipelined form: two T accumulators and two T buffers, the ring behind them, then the
+        // 32 KB of store staging; output accumulators in what tensor memory the T accumulators leave
+        const int64_t stage = plan.stage_bytes, t2 = 2 * static_cast<int64_t>(plan.r_pad) * 256;
+        int64_t ns = (227 * 1024 - 2048 - t2 - 32768) / stage;
+        if (ns > kMaxStages) ns = kMaxStages;
+        if (ns >= 3) {
+            p.num_stages = static_cast<int>(ns);
+            p.staging_off = static_cast<int>(1024 + t2 + ns * stage);
+            p.boxes_per_stage = plan.r_pad / 64;
+            p.acc_base = 2 * plan.r_pad;
+            p.acc_bufs = (512 - 2 * plan.r_pad) / 128;
+            return chain_launch_pipe(grid, static_cast<size_t>(2048 + t2 + ns * stage + 32768), stream, ta, tb1, tb2, to, tt, p);
+        }
+    }
     if (persistent) return chain_launch_multi(grid, plan.smem, stream, ta, tb1, tb2, to, tt, p);
     static bool configured[64] = {};
     int dev = 0;

@@ -486,6 +486,9 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 int chain_launch_act(bool persistent, dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& ta,
                      const CUtensorMap& tb1, const CUtensorMap& tb2, const CUtensorMap& to, const CUtensorMap& tt,
                      const ChainParams& p);
+// Launch of the software-pipelined persistent form (pf_tc_chain_pipe.cuh, compiled in pf_tc_chain_multi.cu).
+int chain_launch_pipe(dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& ta, const CUtensorMap& tb1,
+                      const CUtensorMap& tb2, const CUtensorMap& to, const CUtensorMap& tt, const ChainParams& p);
 // Launch of the persistent form (pf_tc_chain_multi.cu); same arguments as the kernel.
 int chain_launch_multi(dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& ta, const CUtensorMap& tb1,
                        const CUtensorMap& tb2, const CUtensorMap& to, const CUtensorMap& tt, const ChainParams& p);
