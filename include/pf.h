@@ -125,6 +125,20 @@ int pf_lowrank_linear_fwd_act(const void* x, int64_t ldx, const void* U, int64_t
                               int64_t m, int64_t k, int64_t n, int64_t r, int dtype,
                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The step of the backward pass that undoes pf_lowrank_linear_fwd_act's epilogue, before
+ * pf_lowrank_linear_bwd is called with the result: for y = act(z + bias) and an upstream dY [m, n],
+ *   dZ   = dY where y > 0, 0 elsewhere (PF_ACT_RELU);  dZ = dY (PF_ACT_NONE)     written OVER dY
+ *   dbias[j] = sum over the m rows of dZ[:, j]  (plain sum, fp32 accumulation in a fixed order,
+ *              rounded once to `dtype`)                    [n], NULL = not wanted
+ * (Section 2.4: the feed-forward block max(0, x W1 + b1) W2 + b2; biases are trained unfactorized,
+ * Section 2.1.)  y (ldy) is the forward's output and is read only for PF_ACT_RELU.  The workspace of
+ * pf_bias_act_bwd_workspace(m, n) bytes is needed only when dbias is given.  Two launches with
+ * dbias, one without; m = 0 zeroes dbias. */
+size_t pf_bias_act_bwd_workspace(int64_t m, int64_t n);
+int pf_bias_act_bwd(const void* y, int64_t ldy, void* dY, int64_t lddy, void* dbias,
+                    int64_t m, int64_t n, int act, int dtype,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* The same forward for callers that cannot allocate device memory and therefore have no
  * workspace to pass: latency-critical host paths where cudaMalloc is forbidden because it
  * synchronises the device, plug-ins that are handed tensors but no allocator, and processes

@@ -108,6 +108,14 @@ def linear_fwd_act(x, U, V, bias=None, relu=False):
     return y, T
 
 
+def bias_act_bwd(y, dY, relu=True):
+    """Backward of y = act(z + bias) (Section 2.4's max(0, x W1 + b1)): dZ = dY where y > 0 (else 0) for
+    max(0, .), dZ = dY for the identity; dbias = column sums of dZ (plain sums over the rows)."""
+    y, dY = widen(y), widen(dY)
+    dZ = np.where(y > 0, dY, 0.0) if relu else dY.copy()
+    return dZ, dZ.sum(axis=0)
+
+
 def linear_bwd(x, U, V, dY):
     x, U, V, dY = widen(x), widen(U), widen(V), widen(dY)
     m, k = x.shape

@@ -49,6 +49,10 @@ def lib() -> ctypes.CDLL:
         L.pf_lowrank_linear_fwd_act.restype = ci
         L.pf_lowrank_linear_fwd_act.argtypes = [vp, i64, vp, i64, vp, i64, vp, ci, vp, i64, vp, i64,
                                                 i64, i64, i64, i64, ci, vp, sz, vp]
+        L.pf_bias_act_bwd_workspace.restype = sz
+        L.pf_bias_act_bwd_workspace.argtypes = [i64, i64]
+        L.pf_bias_act_bwd.restype = ci
+        L.pf_bias_act_bwd.argtypes = [vp, i64, vp, i64, vp, i64, i64, ci, ci, vp, sz, vp]
         L.pf_lowrank_linear_fwd_static.restype = ci
         L.pf_lowrank_linear_fwd_static.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                                    i64, i64, i64, i64, ci, vp]
@@ -204,6 +208,21 @@ def pf_lowrank_linear_fwd_act(x, U, V, *, bias=None, act=PF_ACT_NONE, y=None, T_
                          (x, U, V, bias, y, T_stash, ws)), out
     _check(lib().pf_lowrank_linear_fwd_act(*args), "pf_lowrank_linear_fwd_act")
     return out
+
+
+def pf_bias_act_bwd(y, dY, *, act=PF_ACT_RELU, want_dbias=True, dbias=None, workspace=None, stream=None):
+    """Backward of y = act(z + bias): dY [m, n] becomes dZ IN PLACE (zeroed where y <= 0 for PF_ACT_RELU);
+    returns dbias [n] (column sums of dZ) or None."""
+    dt = _dtype_code(dY)
+    m, n = dY.shape
+    if dbias is None and want_dbias:
+        dbias = torch.empty((n,), dtype=dY.dtype, device=dY.device)
+    need = int(lib().pf_bias_act_bwd_workspace(m, n)) if dbias is not None else 0
+    ws = _workspace(need, dY.device, workspace, stream)
+    st = lib().pf_bias_act_bwd(_ptr(y), _mat(y, "y") if y is not None else 0, _ptr(dY), _mat(dY, "dY"), _ptr(dbias),
+                               m, n, int(act), dt, _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "pf_bias_act_bwd")
+    return dbias
 
 
 def pf_static_scratch_bytes() -> int:

@@ -224,6 +224,30 @@ int pf_lowrank_linear_fwd_act(const void* x, int64_t ldx, const void* U, int64_t
                            cuda_stream, false, bias, act);
 }
 
+size_t pf_bias_act_bwd_workspace(int64_t m, int64_t n) {
+    if (m <= 0 || n <= 0) return 0;
+    return align_up(static_cast<size_t>(act_bwd_chunks(m)) * n * 4, 256);
+}
+
+int pf_bias_act_bwd(const void* y, int64_t ldy, void* dY, int64_t lddy, void* dbias, int64_t m, int64_t n, int act,
+                    int dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!valid_dtype(dtype) || m < 0 || n < 1) return PF_ERR_INVALID_ARG;
+    if (act != PF_ACT_NONE && act != PF_ACT_RELU) return PF_ERR_INVALID_ARG;
+    if ((m > 0 && !dY) || lddy < n || !elem_aligned(dY, dtype)) return PF_ERR_INVALID_ARG;
+    if (act == PF_ACT_RELU && ((m > 0 && !y) || ldy < n || !elem_aligned(y, dtype))) return PF_ERR_INVALID_ARG;
+    if (dbias && !elem_aligned(dbias, dtype)) return PF_ERR_INVALID_ARG;
+    const size_t need = dbias ? pf_bias_act_bwd_workspace(m, n) : 0;
+    int st = check_ws(workspace, workspace_bytes, need);
+    if (st != PF_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (m == 0) {
+        if (dbias) PF_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(n) * dtype_size(dtype), stream));
+        return PF_OK;
+    }
+    PF_CUDA(act_bwd(y, ldy, dY, lddy, dbias, m, n, act, dtype, static_cast<float*>(workspace), stream));
+    return PF_OK;
+}
+
 int pf_lowrank_linear_bwd(const void* x, int64_t ldx, const void* U, int64_t ldu, const void* V,
                           int64_t ldv, const void* dY, int64_t lddy, const void* T_stash, int64_t ldt,
                           void* dX, int64_t lddx, void* dU, int64_t lddu, void* dV, int64_t lddv,

@@ -103,6 +103,11 @@ struct SliceSums {
     bool out_f32, accumulate;
 };
 cudaError_t slices_to_gradients(const SliceSums* jobs, int count, cudaStream_t stream);
+// Backward of y = act(z + bias): dY becomes dZ in place, db (optional) its column sums.  `part` holds
+// act_bwd_chunks(rows) * cols floats.
+int act_bwd_chunks(int64_t rows);
+cudaError_t act_bwd(const void* y, int64_t ldy, void* dY, int64_t lddy, void* db, int64_t rows, int64_t cols, int act,
+                    int dtype, float* part, cudaStream_t stream);
 // y = act(y + bias) in place: bias [cols] of the storage dtype or null, act 0 = identity, 1 = max(0, .)
 cudaError_t bias_act_inplace(void* y, int64_t ld, int64_t rows, int64_t cols, const void* bias, int act, int dtype,
                              cudaStream_t stream);

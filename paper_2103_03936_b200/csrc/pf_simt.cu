@@ -369,6 +369,67 @@ cudaError_t slices_to_gradients(const SliceSums* jobs, int count, cudaStream_t s
     return cudaGetLastError();
 }
 
+// Backward of y = act(z + bias): dZ = dY where y > 0 (act = max(0, .)) or everywhere (identity), written
+// over dY; partial column sums of dZ per chunk of rows go to `part` [chunks, cols] (fp32), summed in chunk
+// order by the second kernel into db (deterministic).
+template <typename T>
+__global__ void __launch_bounds__(256) act_bwd_kernel(const T* y, int64_t ldy, T* dY, int64_t lddy, int64_t rows,
+                                                      int64_t cols, int act, float* part, int rows_per_chunk) {
+    const int64_t col = static_cast<int64_t>(blockIdx.x) * 32 + (threadIdx.x & 31);
+    const int64_t r_beg = static_cast<int64_t>(blockIdx.y) * rows_per_chunk;
+    const int64_t r_end = r_beg + rows_per_chunk < rows ? r_beg + rows_per_chunk : rows;
+    float sum = 0.f;
+    if (col < cols) {
+        for (int64_t r = r_beg + (threadIdx.x >> 5); r < r_end; r += 8) {
+            float g = static_cast<float>(dY[r * lddy + col]);
+            if (act == 1 && !(static_cast<float>(y[r * ldy + col]) > 0.f)) {
+                g = 0.f;
+                dY[r * lddy + col] = static_cast<T>(0.f);
+            }
+            sum += g;
+        }
+    }
+    __shared__ float red[8][33];
+    red[threadIdx.x >> 5][threadIdx.x & 31] = sum;
+    __syncthreads();
+    if (threadIdx.x < 32 && col < cols && part) {
+        float s = 0.f;
+        for (int w = 0; w < 8; ++w) s += red[w][threadIdx.x];
+        part[static_cast<int64_t>(blockIdx.y) * cols + col] = s;
+    }
+}
+template <typename T>
+__global__ void act_bwd_bias_kernel(const float* part, int chunks, int64_t cols, T* db) {
+    const int64_t col = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (col >= cols) return;
+    float s = 0.f;
+    for (int c = 0; c < chunks; ++c) s += part[static_cast<int64_t>(c) * cols + col];
+    db[col] = static_cast<T>(s);
+}
+int act_bwd_chunks(int64_t rows) {
+    const int64_t c = ceil_div(rows, 256);
+    return static_cast<int>(c < 1 ? 1 : (c > 64 ? 64 : c));
+}
+cudaError_t act_bwd(const void* y, int64_t ldy, void* dY, int64_t lddy, void* db, int64_t rows, int64_t cols, int act,
+                    int dtype, float* part, cudaStream_t stream) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    const int chunks = act_bwd_chunks(rows);
+    const int rpc = static_cast<int>(ceil_div(rows, chunks));
+    const dim3 grid(static_cast<unsigned>(ceil_div(cols, 32)), static_cast<unsigned>(chunks));
+    float* pp = db ? part : nullptr;
+    if (dtype == PF_BF16) {
+        act_bwd_kernel<<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(y), ldy, static_cast<__nv_bfloat16*>(dY), lddy,
+                                                 rows, cols, act, pp, rpc);
+        if (db) act_bwd_bias_kernel<<<static_cast<unsigned>(ceil_div(cols, 256)), 256, 0, stream>>>(part, chunks, cols, static_cast<__nv_bfloat16*>(db));
+    } else {
+        act_bwd_kernel<<<grid, 256, 0, stream>>>(static_cast<const float*>(y), ldy, static_cast<float*>(dY), lddy, rows, cols,
+                                                 act, pp, rpc);
+        if (db) act_bwd_bias_kernel<<<static_cast<unsigned>(ceil_div(cols, 256)), 256, 0, stream>>>(part, chunks, cols, static_cast<float*>(db));
+    }
+    count_launch(db ? 2 : 1);
+    return cudaGetLastError();
+}
+
 // y = act(y + bias) in place (the paths that do not fuse the epilogue into the producing kernel).
 template <typename T>
 __global__ void bias_act_kernel(T* y, int64_t ld, int64_t rows, int64_t cols, const T* bias, int act) {

@@ -97,3 +97,33 @@ def test_bad_arguments():
         pf.pf_lowrank_linear_fwd_act(x, U, V, act=7)
     with pytest.raises(ValueError):
         pf.pf_lowrank_linear_fwd_act(x, U, V, bias=torch.zeros(47, dtype=torch.bfloat16, device="cuda"))
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+@pytest.mark.parametrize("relu", [True, False])
+@pytest.mark.parametrize("m,n,ld_pad", [(1, 1, 0), (77, 50, 3), (700, 264, 0), (4100, 1000, 8), (20000, 33, 0)])
+def test_bias_act_bwd(dtype, relu, m, n, ld_pad):
+    """dZ in place over dY (bit-exact: a copy or a zero), dbias = column sums against the oracle;
+    guard bands and row padding untouched."""
+    y64 = np.maximum(wl.normal(61, 0, (m, n)), 0.0)
+    y_h = wl.round_to(y64, dtype)
+    g_h = wl.round_to(wl.normal(61, 1, (m, n)), dtype)
+    gy = Guarded((m, n), dtype, ld=n + ld_pad if ld_pad else None)
+    gd = Guarded((m, n), dtype, ld=n + ld_pad if ld_pad else None)
+    gb = Guarded((1, n), dtype)
+    gy.t.copy_(dev(y_h, dtype))
+    gd.t.copy_(dev(g_h, dtype))
+    pf.pf_bias_act_bwd(gy.t, gd.t, act=pf.PF_ACT_RELU if relu else pf.PF_ACT_NONE, dbias=gb.t.view(-1))
+    torch.cuda.synchronize()
+    dZ_ref, db_ref = oracle.bias_act_bwd(y_h, g_h, relu=relu)
+    got = oracle.widen(wl.from_torch(gd.t.contiguous(), dtype))
+    np.testing.assert_array_equal(got, dZ_ref)
+    assert_close(gb.t.view(-1), db_ref, dtype, f"dbias {m}x{n} {dtype} relu={relu}", tol=1e-2 if dtype == wl.BF16 else 1e-4)
+    for g in (gy, gd, gb):
+        g.check()
+    # without dbias: one launch, no workspace
+    gd.t.copy_(dev(g_h, dtype))
+    l0 = pf.pf_launch_count()
+    assert pf.pf_bias_act_bwd(gy.t, gd.t, act=pf.PF_ACT_RELU if relu else pf.PF_ACT_NONE, want_dbias=False) is None
+    assert pf.pf_launch_count() - l0 == 1
+    assert pf.pf_last_device_status() == 0

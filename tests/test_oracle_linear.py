@@ -237,3 +237,26 @@ def test_bias_relu_properties():
     # positive homogeneity of max(0, .): scaling x and the bias by 4 (exact in binary) scales y by 4
     y4, _ = oracle.linear_fwd_act(4 * x, U, V, 4 * b, relu=True)
     np.testing.assert_array_equal(y4, 4 * yr)
+
+
+def test_bias_act_bwd_hand_example_and_autograd():
+    """y = max(0, z + b) with y = [[0, 2], [3, 0]] and dY = [[5, 7], [11, 13]]: dZ keeps dY where
+    y > 0 -> [[0, 7], [11, 0]], dbias = column sums [11, 7].  And fp64 autograd of relu(z + b)."""
+    y = np.array([[0.0, 2.0], [3.0, 0.0]], dtype=np.float32)
+    dY = np.array([[5.0, 7.0], [11.0, 13.0]], dtype=np.float32)
+    dZ, db = oracle.bias_act_bwd(y, dY, relu=True)
+    np.testing.assert_array_equal(dZ, [[0.0, 7.0], [11.0, 0.0]])
+    np.testing.assert_array_equal(db, [11.0, 7.0])
+    dZ, db = oracle.bias_act_bwd(y, dY, relu=False)
+    np.testing.assert_array_equal(dZ, dY)
+    np.testing.assert_array_equal(db, [16.0, 20.0])
+    import torch
+    rng = np.random.default_rng(5)
+    z = torch.tensor(rng.standard_normal((9, 6)), dtype=torch.float64, requires_grad=True)
+    b = torch.tensor(rng.standard_normal(6), dtype=torch.float64, requires_grad=True)
+    g = rng.standard_normal((9, 6))
+    out = torch.relu(z + b)
+    out.backward(torch.tensor(g))
+    dZ, db = oracle.bias_act_bwd(out.detach().numpy().astype(np.float32), g.astype(np.float32), relu=True)
+    np.testing.assert_allclose(dZ, z.grad.numpy(), rtol=0, atol=1e-6)
+    np.testing.assert_allclose(db, b.grad.numpy(), rtol=0, atol=1e-5)
