@@ -291,6 +291,14 @@ int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void*
                         int kh, int kw, int stride, int pad, int dtype,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* pf_lowrank_conv_bwd with the gradient options of pf_lowrank_linear_bwd_ex (PF_GRAD_ACCUMULATE,
+ * PF_GRAD_F32) for dU [kh, kw, C, R] and dV [O, R]; same mechanism, same workspace query. */
+int pf_lowrank_conv_bwd_ex(const void* x, const void* U, const void* V, const void* dY,
+                           const void* T_stash, void* dX, void* dU, void* dV,
+                           int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
+                           int pad, int dtype, unsigned flags, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------
  * Flat gradient buffer (Section 4.1 "Implementation details and optimizations": all
  * gradient tensors are packed into one flat buffer so that one all-reduce per iteration

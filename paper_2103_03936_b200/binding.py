@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.pf_lowrank_conv_fwd.argtypes = [vp] * 5 + [ci] * 11 + [vp, sz, vp]
         L.pf_lowrank_conv_bwd.restype = ci
         L.pf_lowrank_conv_bwd.argtypes = [vp] * 8 + [ci] * 11 + [vp, sz, vp]
+        L.pf_lowrank_conv_bwd_ex.restype = ci
+        L.pf_lowrank_conv_bwd_ex.argtypes = [vp] * 8 + [ci] * 11 + [ctypes.c_uint, vp, sz, vp]
         L.pf_pack_factor_grads.restype = ci
         L.pf_pack_factor_grads.argtypes = [vp, vp, ci, ci, vp, i64, vp, vp, sz, vp]
         L.pf_unpack_factor_grads.restype = ci
@@ -393,22 +395,37 @@ def pf_lowrank_conv_fwd(x, U, V, *, stride=1, pad=1, y=None, T_stash=None, want_
 
 
 def pf_lowrank_conv_bwd(x, U, V, dY, *, stride=1, pad=1, T_stash=None, need_dX=True, dX=None,
-                        dU=None, dV=None, workspace=None, stream=None, prepare=False):
-    """Returns (dX or None, dU, dV) for upstream gradient dY [N, Ho, Wo, O]."""
+                        dU=None, dV=None, accumulate=False, grads_f32=False, workspace=None, stream=None,
+                        prepare=False):
+    """Returns (dX or None, dU, dV) for upstream gradient dY [N, Ho, Wo, O].
+    accumulate / grads_f32: as in pf_lowrank_linear_bwd."""
     dt = _dtype_code(x)
     N, H, W, C, R, O, kh, kw, Ho, Wo = _conv_dims(x, U, V, stride, pad)
     if not dY.is_contiguous() or tuple(dY.shape) != (N, Ho, Wo, O):
         raise ValueError("dY must be contiguous [N, Ho, Wo, O]")
     if dX is None and need_dX:
         dX = torch.empty_like(x)
+    flags = (PF_GRAD_ACCUMULATE if accumulate else 0) | (PF_GRAD_F32 if grads_f32 else 0)
+    gdt = torch.float32 if grads_f32 else x.dtype
+    if accumulate and (dU is None or dV is None):
+        raise ValueError("accumulate=True needs the dU and dV to add to")
     if dU is None:
-        dU = torch.empty_like(U)
+        dU = torch.empty(U.shape, dtype=gdt, device=x.device)
     if dV is None:
-        dV = torch.empty_like(V)
+        dV = torch.empty(V.shape, dtype=gdt, device=x.device)
+    if dU.dtype != gdt or dV.dtype != gdt or not dU.is_contiguous() or not dV.is_contiguous():
+        raise ValueError("dU and dV must be contiguous, float32 with grads_f32=True and of x's dtype otherwise")
     ws = _workspace(pf_lowrank_conv_workspace(N, H, W, C, R, O, kh, kw, stride, pad, dt, 1),
                     x.device, workspace, stream)
     args = (_ptr(x), _ptr(U), _ptr(V), _ptr(dY), _ptr(T_stash), _ptr(dX), _ptr(dU), _ptr(dV),
             N, H, W, C, R, O, kh, kw, stride, pad, dt, _ptr(ws), ws.numel(), _stream(stream))
+    if flags:
+        args = args[:19] + (flags,) + args[19:]
+        if prepare:
+            return _Prepared(lib().pf_lowrank_conv_bwd_ex, args, "pf_lowrank_conv_bwd_ex",
+                             (x, U, V, dY, T_stash, dX, dU, dV, ws)), (dX, dU, dV)
+        _check(lib().pf_lowrank_conv_bwd_ex(*args), "pf_lowrank_conv_bwd_ex")
+        return dX, dU, dV
     if prepare:
         return _Prepared(lib().pf_lowrank_conv_bwd, args, "pf_lowrank_conv_bwd",
                          (x, U, V, dY, T_stash, dX, dU, dV, ws)), (dX, dU, dV)

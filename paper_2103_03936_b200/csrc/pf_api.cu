@@ -483,7 +483,7 @@ int pf_lowrank_linear_grouped_bwd(int groups, const void* x, int64_t ldx, int64_
 // ------------------------------------------------------------------------------ conv
 namespace {
 struct ConvWs {
-    size_t off_T, off_dT, off_partial, off_tc, total;
+    size_t off_T, off_dT, off_partial, off_gtmp, off_tc, total;
     int splits_dU, splits_dV;
     int Ho, Wo;
     int64_t P, Pin;
@@ -509,6 +509,8 @@ ConvWs conv_ws(int N, int H, int W, int C, int R, int O, int kh, int kw, int str
         size_t pu = w.splits_dU > 1 ? static_cast<size_t>(w.splits_dU) * Keff * R * 4 : 0;
         size_t pv = w.splits_dV > 1 ? static_cast<size_t>(w.splits_dV) * O * R * 4 : 0;
         w.off_partial = off; off += align_up(pu > pv ? pu : pv, 256);
+        // plain dU and dV of a call that wants them in fp32 or accumulated
+        w.off_gtmp = off; off += align_up(static_cast<size_t>(Keff) * R * s, 256) + align_up(static_cast<size_t>(O) * R * s, 256);
     }
     w.off_tc = off;
     if (dtype == PF_BF16) off += align_up(tc::conv_extra_workspace(N, H, W, C, R, O, kh, kw, stride, pad, bwd), 256);
@@ -584,10 +586,22 @@ int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void*
                         int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
                         int pad, int dtype, void* workspace, size_t workspace_bytes,
                         void* cuda_stream) {
+    return pf_lowrank_conv_bwd_ex(x, U, V, dY, T_stash, dX, dU, dV, N, H, W, C, R, O, kh, kw, stride, pad, dtype, 0u,
+                                  workspace, workspace_bytes, cuda_stream);
+}
+
+int pf_lowrank_conv_bwd_ex(const void* x, const void* U, const void* V, const void* dY,
+                           const void* T_stash, void* dX, void* dU, void* dV,
+                           int N, int H, int W, int C, int R, int O, int kh, int kw, int stride,
+                           int pad, int dtype, unsigned flags, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream) {
     int st = validate_conv_common(x, U, V, N, H, W, C, R, O, kh, kw, stride, pad, dtype);
     if (st != PF_OK) return st;
+    if (flags & ~static_cast<unsigned>(PF_GRAD_ACCUMULATE | PF_GRAD_F32)) return PF_ERR_INVALID_ARG;
+    const bool g_acc = (flags & PF_GRAD_ACCUMULATE) != 0, g_f32 = (flags & PF_GRAD_F32) != 0;
+    const int gdtype = g_f32 ? PF_F32 : dtype;
     if ((!dY && N > 0) || !dU || !dV) return PF_ERR_INVALID_ARG;
-    if (!elem_aligned(dY, dtype) || !elem_aligned(dU, dtype) || !elem_aligned(dV, dtype) ||
+    if (!elem_aligned(dY, dtype) || !elem_aligned(dU, gdtype) || !elem_aligned(dV, gdtype) ||
         (dX && !elem_aligned(dX, dtype)) || (T_stash && !elem_aligned(T_stash, dtype)))
         return PF_ERR_INVALID_ARG;
     const ConvWs w = conv_ws(N, H, W, C, R, O, kh, kw, stride, pad, dtype, true);
@@ -597,12 +611,39 @@ int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void*
     const size_t s = dtype_size(dtype);
     const int64_t Keff = static_cast<int64_t>(kh) * kw * C;
     if (w.P == 0) {
-        PF_CUDA(cudaMemsetAsync(dU, 0, Keff * R * s, stream));
-        PF_CUDA(cudaMemsetAsync(dV, 0, static_cast<size_t>(O) * R * s, stream));
+        if (!g_acc) {
+            PF_CUDA(cudaMemsetAsync(dU, 0, Keff * R * dtype_size(gdtype), stream));
+            PF_CUDA(cudaMemsetAsync(dV, 0, static_cast<size_t>(O) * R * dtype_size(gdtype), stream));
+        }
         if (dX && w.Pin > 0) PF_CUDA(cudaMemsetAsync(dX, 0, w.Pin * C * s, stream));
         return PF_OK;
     }
     char* ws = static_cast<char*>(workspace);
+    // with gradient flags: plain dU, dV into the workspace, then one pass into the caller's matrices
+    void* const user_dU = dU;
+    void* const user_dV = dV;
+    if (flags) {
+        dU = ws + w.off_gtmp;
+        dV = ws + w.off_gtmp + align_up(static_cast<size_t>(Keff) * R * s, 256);
+    }
+    tc::LinearArgs::Slices su_info, sv_info;
+    auto finish = [&]() -> int {
+        if (!flags) return PF_OK;
+        SliceSums jobs[2];
+        int nj = 0;
+        if (su_info.splits > 1)
+            jobs[nj++] = SliceSums{su_info.partial, user_dU, R, static_cast<int>(Keff), R, su_info.splits, su_info.bn,
+                                   su_info.tiles_x, su_info.tiles_y, g_f32, g_acc};
+        else
+            PF_CUDA(grad_combine(user_dU, R, gdtype, dU, R, dtype, Keff, R, g_acc, stream));
+        if (sv_info.splits > 1)
+            jobs[nj++] = SliceSums{sv_info.partial, user_dV, R, O, R, sv_info.splits, sv_info.bn, sv_info.tiles_x,
+                                   sv_info.tiles_y, g_f32, g_acc};
+        else
+            PF_CUDA(grad_combine(user_dV, R, gdtype, dV, R, dtype, O, R, g_acc, stream));
+        if (nj) PF_CUDA(slices_to_gradients(jobs, nj, stream));
+        return PF_OK;
+    };
 
     if (dtype == PF_BF16) {
         tc::ConvArgs a;
@@ -612,9 +653,13 @@ int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void*
         a.N = N; a.H = H; a.W = W; a.C = C; a.R = R; a.O = O; a.kh = kh; a.kw = kw;
         a.stride = stride; a.pad = pad; a.Ho = w.Ho; a.Wo = w.Wo;
         a.ws = ws + w.off_tc; a.ws_T = ws + w.off_T; a.ws_G = ws + w.off_dT; a.stream = stream;
+        a.du_slices = &su_info; a.dv_slices = &sv_info;
         int handled = 0;
         st = tc::conv_bwd(a, &handled);
-        if (st != PF_OK || handled) return st;
+        if (st != PF_OK) return st;
+        if (handled) return finish();
+        su_info = tc::LinearArgs::Slices();
+        sv_info = tc::LinearArgs::Slices();
     }
     MatA Aim;
     std::memset(&Aim, 0, sizeof(Aim));
@@ -640,7 +685,7 @@ int pf_lowrank_conv_bwd(const void* x, const void* U, const void* V, const void*
         Bt.p = U; Bt.kind = B_TAPSPLIT; Bt.l_fast = 1; Bt.R = R; Bt.CR = C * R;
         PF_CUDA(simt_gemm(mk(Ac, Bt, dX, C, w.Pin, C, static_cast<int64_t>(kh) * kw * R, dtype), stream));
     }
-    return PF_OK;
+    return finish();
 }
 
 // ------------------------------------------------------------------------------ pack

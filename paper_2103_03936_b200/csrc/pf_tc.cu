@@ -1393,6 +1393,18 @@ int conv_bwd(const ConvArgs& a, int* handled) {
     if (st == PF_ERR_UNSUPPORTED) return PF_OK;      // declined: nothing has been launched
     if (st != PF_OK) return st;
     *handled = 1;
+    {   // both reductions are launched exactly as prepared (together or one by one)
+        const GemmLaunch* gs[2] = {&gu, &gv};
+        LinearArgs::Slices* outs[2] = {a.du_slices, a.dv_slices};
+        for (int i = 0; i < 2; ++i) {
+            if (!outs[i]) continue;
+            *outs[i] = LinearArgs::Slices();
+            if (gs[i]->p.splits > 1) {
+                outs[i]->partial = gs[i]->p.partial; outs[i]->splits = gs[i]->p.splits; outs[i]->bn = gs[i]->bn;
+                outs[i]->tiles_x = static_cast<int>(gs[i]->grid.x); outs[i]->tiles_y = static_cast<int>(gs[i]->grid.y);
+            }
+        }
+    }
     if (!a.T) {   // recompute the thin convolution (phase 1 of the forward only)
         const ChainConv cv{a.N, a.H, a.W, a.C, a.kh, a.kw, a.pad};
         st = chain(a.x, a.C, M, Keff, a.U, a.R, a.R, a.V, a.R, a.O, nullptr, a.O, a.ws_T, a.R, a.stream, &cv);

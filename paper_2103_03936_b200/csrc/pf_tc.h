@@ -38,6 +38,8 @@ struct ConvArgs {
     int N, H, W, C, R, O, kh, kw, stride, pad, Ho, Wo;
     char *ws, *ws_T, *ws_G;
     cudaStream_t stream;
+    // backward: where the fp32 slices of dU / dV were left (see LinearArgs::Slices); may be null
+    LinearArgs::Slices *du_slices, *dv_slices;
 };
 
 // Fused chain kernel (pf_tc_chain.cu): out = (A * B1) * B2^T with the intermediate on chip.

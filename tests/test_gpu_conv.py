@@ -155,3 +155,31 @@ def test_empty_batch():
     _, dU, dV = pf.pf_lowrank_conv_bwd(x, U, V, torch.empty((0, 8, 8, 8), dtype=torch.bfloat16, device="cuda"))
     torch.cuda.synchronize()
     assert torch.all(dU == 0) and torch.all(dV == 0)
+
+
+@pytest.mark.parametrize("dtype,N,H,W,C,R,O,stride", [(wl.BF16, 4, 16, 16, 128, 64, 128, 1), (wl.BF16, 2, 8, 8, 24, 8, 16, 2),
+                                                      (wl.F32, 2, 8, 8, 16, 8, 24, 1)])
+def test_conv_grads_fp32_and_accumulated(dtype, N, H, W, C, R, O, stride):
+    """pf_lowrank_conv_bwd_ex: fp32 factor gradients reproduce the plain call when rounded (same sums),
+    and accumulation over two halves of the batch gives the whole batch's gradient on top of the
+    previous contents; tensor-core envelope, FMA kernels (stride 2), fp32 storage."""
+    c = wl.ConvCase("cg", N, H, W, C, R, O, dtype, 71, stride=stride)
+    d = c.generate()
+    x, U, V, dY = (dev(d[k_], dtype) for k_ in ("x", "U", "V", "dY"))
+    _, dU0, dV0 = pf.pf_lowrank_conv_bwd(x, U, V, dY, stride=stride, need_dX=False)
+    _, dU1, dV1 = pf.pf_lowrank_conv_bwd(x, U, V, dY, stride=stride, need_dX=False, grads_f32=True)
+    assert dU1.dtype == torch.float32 and torch.equal(dU1.to(dU0.dtype), dU0) and torch.equal(dV1.to(dV0.dtype), dV0)
+    _, dU_ref, dV_ref = oracle.conv_bwd(d["x"], d["U"], d["V"], d["dY"], stride=stride, pad=1)
+    tol = 1e-2 if dtype == wl.BF16 else 1e-4
+    assert_close(dU1, dU_ref, wl.F32, "conv fp32 dU", tol=tol)
+    assert_close(dV1, dV_ref, wl.F32, "conv fp32 dV", tol=tol)
+    prevU = torch.full(U.shape, 0.25, dtype=torch.float32, device="cuda")
+    prevV = torch.full(V.shape, -0.5, dtype=torch.float32, device="cuda")
+    h = N // 2
+    for lo, hi in ((0, h), (h, N)):
+        pf.pf_lowrank_conv_bwd(x[lo:hi], U, V, dY[lo:hi], stride=stride, need_dX=False, dU=prevU, dV=prevV,
+                               accumulate=True, grads_f32=True)
+    torch.cuda.synchronize()
+    assert_close(prevU, 0.25 + dU_ref, wl.F32, "conv accumulated dU", tol=tol)
+    assert_close(prevV, -0.5 + dV_ref, wl.F32, "conv accumulated dV", tol=tol)
+    assert pf.pf_last_device_status() == 0
