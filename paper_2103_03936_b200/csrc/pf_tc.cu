@@ -1323,10 +1323,12 @@ void reset_fix_counters() {
 
 // Tensor-core envelope of the factorized convolution: stride 1, "same" padding, channel counts
 // that tile evenly, image rows that pack into 128-pixel (forward, dX) and 64-pixel (dU) tiles.
-static bool conv_tc_ok(const ConvArgs& a) {
-    if (a.stride != 1 || a.kh != a.kw || 2 * a.pad != a.kh - 1) return false;
+// (The forward also takes stride 2: its image tiles are fetched with a step of two pixels, and only the
+// output row has to fit a tile.  The backward of a strided convolution runs on the FMA kernels.)
+static bool conv_tc_ok(const ConvArgs& a, bool fwd = false) {
+    if ((a.stride != 1 && !(fwd && a.stride == 2)) || a.kh != a.kw || 2 * a.pad != a.kh - 1) return false;
     if (a.C % 128 != 0 || a.R % 64 != 0 || a.O % 8 != 0 || a.R > 384) return false;
-    if (a.W > 64) return false;                       // one image row must fit a 64-pixel k-block of dU
+    if (fwd ? a.Wo > 128 : a.W > 64) return false;    // backward: one image row must fit a 64-pixel k-block of dU
     if (static_cast<int64_t>(a.N) * a.H * a.W > 0x7fffffff) return false;
     return encode_fn() != nullptr;
 }
@@ -1345,14 +1347,15 @@ size_t conv_extra_workspace(int N, int H, int W, int C, int R, int O, int kh, in
 
 int conv_fwd(const ConvArgs& a, int* handled) {
     *handled = 0;
-    if (!conv_tc_ok(a) || !aligned16(a.x) || !aligned16(a.U) || !aligned16(a.V) || !aligned16(a.y) ||
+    if (!conv_tc_ok(a, true) || !aligned16(a.x) || !aligned16(a.U) || !aligned16(a.V) || !aligned16(a.y) ||
         (a.T && !aligned16(a.T)))
         return PF_OK;
-    const int64_t M = static_cast<int64_t>(a.N) * a.H * a.W, Keff = static_cast<int64_t>(a.kh) * a.kw * a.C;
+    const int64_t M = static_cast<int64_t>(a.N) * a.Ho * a.Wo, Keff = static_cast<int64_t>(a.kh) * a.kw * a.C;
+    if (M < 1 || a.stride * a.Wo > 256) return PF_OK;
     ChainPlan plan;
-    if (!chain_plan(M, Keff, a.O, a.R, true, &plan)) return PF_OK;
+    if (!chain_plan(M, Keff, a.O, a.R, true, &plan, conv_box_h(a.Ho, a.Wo, 128) * a.Wo)) return PF_OK;
     *handled = 1;
-    const ChainConv cv{a.N, a.H, a.W, a.C, a.kh, a.kw, a.pad};
+    const ChainConv cv{a.N, a.H, a.W, a.C, a.kh, a.kw, a.pad, a.stride};
     return chain(a.x, a.C, M, Keff, a.U, a.R, a.R, a.V, a.R, a.O, a.y, a.O, a.T, a.R, a.stream, &cv);
 }
 

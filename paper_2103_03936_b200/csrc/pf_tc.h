@@ -53,8 +53,11 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
 int conv_box_h(int H, int W, int limit);
 // When `conv` is given, A is an NHWC image and phase 1 is the implicit GEMM of a kh x kw, stride-1,
 // "same"-padded convolution: M = N*H*W pixels, K1 = kh*kw*C, B1 = U as a (kh*kw*C) x r matrix.
+// stride (1 or 2) applies to the k x k convolution: M = N*Ho*Wo output pixels, and the image tile of a tap
+// is fetched with that step between pixels (a tensor map with element strides).
 struct ChainConv {
     int N, H, W, C, kh, kw, pad;
+    int stride = 1;
 };
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,

@@ -54,17 +54,39 @@ bool chain_plan(int64_t M, int64_t K1, int64_t N2, int64_t r, bool has_out, Chai
     return true;
 }
 
+// NHWC image map whose boxes take every `stride`-th pixel along W and H: box_w x box_h pixels of 64
+// channels are loaded (the box extents are given in traversed elements, i.e. times the stride).
+static bool make_map_nhwc_strided(CUtensorMap* map, const void* p, int64_t N, int64_t H, int64_t W, int64_t C, int box_w,
+                                  int box_h, int stride) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
+                                static_cast<cuuint64_t>(N)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 2, static_cast<cuuint64_t>(W) * C * 2,
+                                   static_cast<cuuint64_t>(H) * W * C * 2};
+    const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(box_w * stride), static_cast<cuuint32_t>(box_h * stride), 1u};
+    const cuuint32_t estr[4] = {1u, static_cast<cuuint32_t>(stride), static_cast<cuuint32_t>(stride), 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(p), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // out may be null (phase 1 only: T is written and nothing else).  All pointers must satisfy tma_ok.
 int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int64_t ldb1, int64_t r,
           const void* B2, int64_t ldb2, int64_t N2, void* out, int64_t ldo, void* T, int64_t ldt,
           cudaStream_t stream, const ChainConv* conv, int max_split, const void* bias, int act) {
     ChainPlan plan;
-    const int box_h = conv ? conv_box_h(conv->H, conv->W, 128) : 1;
-    const int rows_tile = conv ? box_h * conv->W : 128;
+    const int cs = conv ? conv->stride : 1;
+    const int Ho = conv ? (conv->H + 2 * conv->pad - conv->kh) / cs + 1 : 1;
+    const int Wo = conv ? (conv->W + 2 * conv->pad - conv->kw) / cs + 1 : 1;
+    const int box_h = conv ? conv_box_h(Ho, Wo, 128) : 1;          // output rows of one tile
+    const int rows_tile = conv ? box_h * Wo : 128;
+    if (conv && (Wo > 128 || cs * Wo > 256 || cs * box_h > 256)) return PF_ERR_UNSUPPORTED;
     if (!chain_plan(M, K1, N2, r, out != nullptr, &plan, rows_tile, max_split)) return PF_ERR_UNSUPPORTED;
     CUtensorMap ta, tb1, tb2, to, tt;
-    bool ok = conv ? cached_map_nhwc(&ta, A, conv->N, conv->H, conv->W, conv->C, conv->W, box_h)
-                   : cached_map_2d(&ta, A, M, K1, lda, 128);
+    bool ok = !conv ? cached_map_2d(&ta, A, M, K1, lda, 128)
+              : cs == 1 ? cached_map_nhwc(&ta, A, conv->N, conv->H, conv->W, conv->C, conv->W, box_h)
+                        : make_map_nhwc_strided(&ta, A, conv->N, conv->H, conv->W, conv->C, Wo, box_h, cs);
     ok = ok && cached_map_2d(&tb1, B1, K1, r, ldb1, 64) && cached_map_2d(&tb2, B2, N2, r, ldb2, 128);
     if (conv) {   // outputs seen as [tiles][rows_tile][cols] so that partial tiles are clipped per tile
         ok = ok && (out ? cached_map_tiled_rows(&to, out, M / rows_tile, rows_tile, N2, 32)
@@ -84,7 +106,8 @@ int chain(const void* A, int64_t lda, int64_t M, int64_t K1, const void* B1, int
     p.conv_cblks = 0; p.conv_kw = 1; p.conv_pad = 0; p.conv_box_h = 1; p.conv_tiles_per_img = 1;
     if (conv) {
         p.conv_cblks = conv->C / 64; p.conv_kw = conv->kw; p.conv_pad = conv->pad;
-        p.conv_box_h = box_h; p.conv_tiles_per_img = conv->H / box_h;
+        // the kernel places tile i of an image at input row i * conv_box_h - pad: stride x the output rows
+        p.conv_box_h = box_h * cs; p.conv_tiles_per_img = Ho / box_h;
     }
     p.rows_tile = rows_tile;
     p.row_tiles = plan.row_tiles;

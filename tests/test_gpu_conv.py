@@ -183,3 +183,28 @@ def test_conv_grads_fp32_and_accumulated(dtype, N, H, W, C, R, O, stride):
     assert_close(prevU, 0.25 + dU_ref, wl.F32, "conv accumulated dU", tol=tol)
     assert_close(prevV, -0.5 + dV_ref, wl.F32, "conv accumulated dV", tol=tol)
     assert pf.pf_last_device_status() == 0
+
+
+@pytest.mark.parametrize("N,H,W,C,R,O", [(4, 16, 16, 128, 64, 128), (3, 14, 14, 256, 64, 256), (2, 15, 17, 128, 128, 72),
+                                         (40, 32, 32, 128, 64, 256)])
+def test_stride2_forward_on_tensor_cores(N, H, W, C, R, O):
+    """Stride-2 3 x 3 convolutions (the first convolution of a ResNet stage): the forward runs on the fused
+    tensor-core kernel with image tiles fetched two pixels apart (one launch; even and odd image sizes,
+    output rows that do not fill a tile, more tiles than SMs); the backward runs on the FMA kernels."""
+    c = wl.ConvCase("s2", N, H, W, C, R, O, wl.BF16, 81, stride=2)
+    d = c.generate()
+    x, U, V = (dev(d[k_], wl.BF16) for k_ in ("x", "U", "V"))
+    gy = Guarded((N, c.Ho, c.Wo, O), wl.BF16)
+    gT = Guarded((N, c.Ho, c.Wo, R), wl.BF16)
+    l0 = pf.pf_launch_count()
+    pf.pf_lowrank_conv_fwd(x, U, V, stride=2, pad=1, y=gy.t, T_stash=gT.t)
+    assert pf.pf_launch_count() - l0 == 1
+    torch.cuda.synchronize()
+    y_ref, T_ref = oracle.conv_fwd(d["x"], d["U"], d["V"], 2, 1)
+    assert_close(gy.t, y_ref, wl.BF16, "stride-2 y")
+    assert_close(gT.t, T_ref, wl.BF16, "stride-2 T")
+    assert_blocks_close(gy.t, y_ref, wl.BF16, "stride-2 y", br=32)
+    gy.check()
+    gT.check()
+    assert pf.pf_last_device_status() == 0
+    run_conv(c)          # and the whole forward + backward against the oracle
